@@ -1,0 +1,194 @@
+/*
+ * prepack-b200: C ABI of the prepacked-prefill attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library follows Algorithm 1 ("Prepacking") of arXiv 2404.09529:
+ *   line 4   BINPACK            -> pp_pack                 (host)
+ *   line 5   TENSORIZE          -> layout contract below   (no call)
+ *   line 6   INDEPENDENT-MASK   -> applied inside pp_prefill_attention, never materialised
+ *   line 7   RESTART-PE         -> applied inside pp_prefill_attention (rotary), also
+ *                                  available as explicit ids from pp_fill_position_ids
+ *   line 8   forward + UNPACK   -> pp_prefill_attention (the attention of one layer) and
+ *                                  pp_unpack_kv
+ *
+ * Conventions
+ *   - Every function returns an int status (PP_OK = 0, errors < 0). Nothing aborts or throws.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA global memory of the
+ *     current device. The library never allocates device memory; callers own every buffer.
+ *   - Streams are passed as void* (a cudaStream_t); NULL is the default stream. Device work is
+ *     enqueued on that stream and the call returns without synchronising unless stated.
+ *   - Tensors are bf16. Packed tensors are dense [R, M, H, D] (bins, rows per bin = capacity,
+ *     heads, head_dim), row t of bin b being the token at bin-local offset t (TENSORIZE,
+ *     Section 3.1: bins are tail-padded to the bin size). Rows at or after the bin's used
+ *     length are padding: they must hold finite values (zeros are fine) and their outputs are
+ *     unspecified.
+ *   - Packing arrays are int32, "segments" are prompts in bin-major placement order.
+ */
+#ifndef PREPACK_B200_PP_H_
+#define PREPACK_B200_PP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  PP_OK = 0,
+  PP_ERR_INVALID_ARG = -1,      /* null pointer, k < 1, inconsistent packing arrays            */
+  PP_ERR_LENGTH = -2,           /* a prompt length < 1 or > capacity                          */
+  PP_ERR_BUFFER_TOO_SMALL = -3, /* workspace / arena smaller than the *_bytes query            */
+  PP_ERR_UNSUPPORTED = -4,      /* head_dim not in {64,128}, Hq % Hkv != 0, device not sm_100  */
+  PP_ERR_ALIGNMENT = -5,        /* a device tensor pointer is not 16-byte aligned              */
+  PP_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed (see pp_last_cuda_error)  */
+  PP_ERR_DEVICE_TIMEOUT = -7,   /* a bounded device-side wait gave up (device status word)     */
+  PP_ERR_NO_MEMORY = -8         /* host allocation failed                                      */
+};
+
+/* Flags for pp_attn_params.flags */
+enum {
+  PP_FLAG_SKIP_ROPE = 1,  /* q and k already carry the rotary encoding: run attention only     */
+  PP_FLAG_ROPE_ONLY = 2   /* apply the restart rotary encoding to q and k, skip attention      */
+};
+
+typedef struct pp_attn_params {
+  int32_t n_q_heads;     /* Hq                                                                 */
+  int32_t n_kv_heads;    /* Hkv, divides Hq; query head h reads KV head h / (Hq / Hkv)          */
+  int32_t head_dim;      /* D: 64 or 128                                                       */
+  float rope_base;       /* rotary base; theta_j = base^(-2j/D), pairs (j, j + D/2)             */
+  float softmax_scale;   /* 0 selects 1/sqrt(D) (Section 2.1)                                  */
+  int32_t capacity;      /* M: rows per bin (Algorithm 1 line 3: the longest prompt)           */
+  int32_t n_bins;        /* R                                                                  */
+  int32_t flags;         /* PP_FLAG_* or 0                                                     */
+} pp_attn_params;
+
+/* Library version (major * 10000 + minor * 100 + patch). */
+int pp_version(void);
+/* Static, never-NULL description of a status code. */
+const char* pp_strerror(int status);
+/* Text of the last CUDA error seen by the calling thread inside the library ("" if none). */
+const char* pp_last_cuda_error(void);
+
+/*
+ * BINPACK -- Section 3.1 and Algorithm 1 lines 2-4. Host only, deterministic.
+ * First-fit-decreasing of k prompt lengths into bins of `capacity` rows (0 selects the longest
+ * prompt, the paper's choice). Items are taken by length descending, equal lengths by original
+ * index ascending; each goes to the lowest-numbered bin with room, else opens a new bin; bins
+ * are numbered in creation order and keep their items in placement order.
+ * Outputs (caller-allocated host arrays; any may be NULL to skip it except n_bins):
+ *   n_bins       [1]    r
+ *   capacity_out [1]    the capacity used
+ *   bin_seg_ptr  [k+1]  CSR over segments; entries 0..r are written
+ *   seg_prompt   [k]    original prompt index of each segment
+ *   seg_start    [k]    bin-local start row of each segment (the paper's idx)
+ *   seg_len      [k]    length of each segment
+ *   bin_of,off_of[k]    inverse map, original prompt order: prompt i lives in bin bin_of[i] at
+ *                       rows off_of[i] .. off_of[i]+lengths[i]-1
+ * Errors: PP_ERR_INVALID_ARG (NULL lengths/n_bins, k < 1), PP_ERR_LENGTH, PP_ERR_NO_MEMORY.
+ */
+int pp_pack(const int32_t* lengths, int32_t k, int32_t capacity,
+            int32_t* n_bins, int32_t* capacity_out,
+            int32_t* bin_seg_ptr, int32_t* seg_prompt, int32_t* seg_start, int32_t* seg_len,
+            int32_t* bin_of, int32_t* off_of);
+
+/*
+ * RESTART-PE as explicit ids -- Section 3.2, Algorithm 1 line 7. Host only.
+ * position_ids [n_bins*capacity]: 0,1,2,... restarting at every segment start; padding rows 0.
+ * segment_ids  [n_bins*capacity]: index into the seg_* arrays; padding rows -1. Either output
+ * may be NULL. Errors: PP_ERR_INVALID_ARG on NULL inputs or segments that do not tile a bin
+ * contiguously from row 0 within `capacity`.
+ */
+int pp_fill_position_ids(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
+                         const int32_t* seg_start, const int32_t* seg_len,
+                         int32_t* position_ids, int32_t* segment_ids);
+
+/*
+ * Bytes of workspace pp_prefill_attention needs, for a batch of k prompts packed as `params`
+ * says (same size for the device workspace and for the host staging buffer). 0 on bad input.
+ */
+size_t pp_prefill_workspace_bytes(const pp_attn_params* params, int32_t k);
+
+/*
+ * Prefill attention over the packed batch -- Algorithm 1 lines 6-8 for one attention layer:
+ * restart rotary encoding of q and k (Section 3.2), then per bin and query head
+ *   o_i = sum_j softmax_j(q'_i . k'_j * scale) v_j   over keys j of the SAME prompt with j <= i
+ * (independent mask M' of Section 3.2: a lower-triangular block per prompt span, zero elsewhere).
+ *
+ *   params                         shapes, see pp_attn_params
+ *   bin_seg_ptr, seg_start, seg_len, k
+ *                                  host packing arrays from pp_pack (k = number of segments)
+ *   q   device [R, M, Hq,  D] bf16 in/out: overwritten with the rotated queries
+ *   k_  device [R, M, Hkv, D] bf16 in/out: overwritten with the rotated keys (this is the
+ *                                  packed K cache that pp_unpack_kv reads)
+ *   v   device [R, M, Hkv, D] bf16 read only
+ *   o   device [R, M, Hq,  D] bf16 out; padding rows unspecified
+ *   workspace       device, >= pp_prefill_workspace_bytes, 16-byte aligned; holds the segment
+ *                   table and the tile work list for the duration of the enqueued work
+ *   host_workspace  host, same size (pinned memory keeps the call asynchronous); the library
+ *                   builds the tables here and copies them with one async H2D on `stream`; it
+ *                   must stay untouched until that copy has run
+ *   device_status   device int32 or NULL; set non-zero by the kernel if a bounded wait inside
+ *                   it gave up (then outputs are invalid). The caller zeroes and reads it.
+ * Arithmetic: rotation in fp32 with one rounding to bf16; scores and outputs accumulated in
+ * fp32 on the tensor cores, probabilities rounded to bf16 before the P.V product.
+ * Errors (all detected before anything is enqueued): PP_ERR_INVALID_ARG, PP_ERR_LENGTH,
+ * PP_ERR_UNSUPPORTED, PP_ERR_ALIGNMENT, PP_ERR_BUFFER_TOO_SMALL; PP_ERR_CUDA from launches.
+ */
+int pp_prefill_attention(const pp_attn_params* params,
+                         const int32_t* bin_seg_ptr, const int32_t* seg_start,
+                         const int32_t* seg_len, int32_t k,
+                         void* q, void* k_, const void* v, void* o,
+                         void* workspace, void* host_workspace, size_t workspace_bytes,
+                         int32_t* device_status, void* stream);
+
+/* Bytes of workspace pp_unpack_kv needs for k prompts (device and host staging alike). */
+size_t pp_unpack_workspace_bytes(int32_t k);
+
+/*
+ * UNPACK -- Algorithm 1 line 8, Section 4.3: copy each prompt's rotated keys and its values out
+ * of the packed tensors into that prompt's own cache, in original prompt order.
+ *   cache[i][h][p][:] = packed[bin_of[i], off_of[i] + p, h, :]   for p < lengths[i]
+ *   bin_of, off_of, lengths  host [k], original prompt order (lengths may be shorter than the
+ *                            packed segment, e.g. in padded mode; only that many rows are copied)
+ *   k_rot, v       device [R, M, Hkv, D] bf16 (k_rot = the k_ tensor after pp_prefill_attention)
+ *   k_cache, v_cache device bf16 pools; prompt i's block starts at element cache_off[i] and is
+ *                  laid out [Hkv, cache_cap[i], D]; rows >= lengths[i] are left untouched
+ *   cache_off      host int64 [k], multiples of 8 elements; cache_cap host int32 [k] >= lengths
+ *   workspace / host_workspace  >= pp_unpack_workspace_bytes(k), as for pp_prefill_attention
+ * Pure copy, bit exact. Errors: PP_ERR_INVALID_ARG, PP_ERR_LENGTH, PP_ERR_ALIGNMENT,
+ * PP_ERR_BUFFER_TOO_SMALL, PP_ERR_UNSUPPORTED, PP_ERR_CUDA.
+ */
+int pp_unpack_kv(const pp_attn_params* params,
+                 const int32_t* bin_of, const int32_t* off_of, const int32_t* lengths, int32_t k,
+                 const void* k_rot, const void* v, void* k_cache, void* v_cache,
+                 const int64_t* cache_off, const int32_t* cache_cap,
+                 void* workspace, void* host_workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Whole path from host memory (Algorithm 1 lines 2-8 for one attention layer), for callers whose
+ * tensors live on the host. Packs `lengths` (pp_pack, capacity = longest prompt), lays the
+ * prompts out as the packed batch on the device (TENSORIZE: one H2D copy per prompt and tensor,
+ * padding rows zeroed), runs pp_prefill_attention and pp_unpack_kv there, copies the outputs
+ * back and synchronises `stream` before returning.
+ *   params                   n_q_heads, n_kv_heads, head_dim, rope_base, softmax_scale are
+ *                            read; capacity and n_bins are filled in from the packing
+ *   q_host                   host bf16 [T, Hq, D], tokens of prompt 0, then prompt 1, ...
+ *   k_host, v_host           host bf16 [T, Hkv, D], same order (T = sum of lengths)
+ *   o_host                   host out bf16 [T, Hq, D], same order
+ *   k_cache_host, v_cache_host host out bf16; prompt i at element Hkv*D*(sum of earlier
+ *                            lengths), laid out [Hkv, lengths[i], D]
+ *   arena, arena_bytes       device scratch >= pp_prefill_host_arena_bytes(params, lengths, k),
+ *                            256-byte aligned
+ * Pinned host buffers give full copy bandwidth; pageable ones work too.
+ * Errors: as the three calls it is made of, plus PP_ERR_DEVICE_TIMEOUT.
+ */
+size_t pp_prefill_host_arena_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k);
+int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, int32_t k,
+                    const void* q_host, const void* k_host, const void* v_host,
+                    void* o_host, void* k_cache_host, void* v_cache_host,
+                    void* arena, size_t arena_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PREPACK_B200_PP_H_ */

@@ -1,0 +1,19 @@
+"""prepack-b200: prefill attention over bin-packed prompts on NVIDIA B200 (sm_100a).
+
+Thin Python binding over the C-ABI library declared in ``include/pp.h``; every step of
+the path (packing, restart rotary encoding, packed attention, KV unpack) runs inside that
+library. PyTorch is used by callers only for device memory and streams.
+"""
+from .binding import (PP_FLAG_ROPE_ONLY, PP_FLAG_SKIP_ROPE, AttnParams, Packing, PrepackError,
+                      Workspaces, lib_path, load_library, pp_fill_position_ids,
+                      pp_last_cuda_error, pp_pack, pp_prefill_attention, pp_prefill_host,
+                      pp_prefill_host_arena_bytes, pp_prefill_workspace_bytes, pp_strerror,
+                      pp_unpack_kv, pp_unpack_workspace_bytes, pp_version)
+
+__all__ = [
+    "PP_FLAG_ROPE_ONLY", "PP_FLAG_SKIP_ROPE", "AttnParams", "Packing", "PrepackError", "Workspaces",
+    "lib_path", "load_library", "pp_fill_position_ids", "pp_last_cuda_error", "pp_pack",
+    "pp_prefill_attention", "pp_prefill_host", "pp_prefill_host_arena_bytes",
+    "pp_prefill_workspace_bytes", "pp_strerror", "pp_unpack_kv", "pp_unpack_workspace_bytes",
+    "pp_version",
+]

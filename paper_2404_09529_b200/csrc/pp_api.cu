@@ -1,0 +1,275 @@
+// C-ABI entry points that touch the device: argument validation, table upload, kernel launches.
+// Algorithm 1 lines 5-8 of the prepacking paper; see include/pp.h for the contracts.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "pp_internal.h"
+
+namespace pp {
+
+static thread_local char g_cuda_error[256] = "";
+
+int note_cuda_error(int cuda_error, const char* what) {
+  const char* txt = cuda_error >= 0 ? cudaGetErrorString((cudaError_t)cuda_error) : "n/a";
+  std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%d)", what, txt, cuda_error);
+  return PP_ERR_CUDA;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_params(const pp_attn_params* p) {
+  if (!p) return PP_ERR_INVALID_ARG;
+  if (p->n_q_heads < 1 || p->n_kv_heads < 1 || p->capacity < 1 || p->n_bins < 1) return PP_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return PP_ERR_UNSUPPORTED;
+  if (p->n_q_heads % p->n_kv_heads != 0) return PP_ERR_UNSUPPORTED;
+  if (p->n_kv_heads > 65535) return PP_ERR_UNSUPPORTED;
+  if (!(p->rope_base > 0.f) || p->softmax_scale < 0.f) return PP_ERR_INVALID_ARG;
+  return PP_OK;
+}
+
+// The kernels are built for sm_100a only.
+int check_device() {
+  static thread_local int cached_dev = -1;
+  static thread_local int cached_status = PP_OK;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return note_cuda_error((int)e, "cudaGetDevice");
+  if (dev == cached_dev) return cached_status;
+  int major = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) return note_cuda_error((int)e, "cudaDeviceGetAttribute");
+  cached_dev = dev;
+  cached_status = (major == 10) ? PP_OK : PP_ERR_UNSUPPORTED;
+  return cached_status;
+}
+
+}  // namespace
+}  // namespace pp
+
+extern "C" const char* pp_last_cuda_error(void) { return pp::g_cuda_error; }
+
+extern "C" size_t pp_prefill_workspace_bytes(const pp_attn_params* params, int32_t k) {
+  if (pp::check_params(params) != PP_OK || k < 1) return 0;
+  return sizeof(int32_t) * pp::prefill_table_ints(params->n_bins, params->capacity, k);
+}
+
+extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t* bin_seg_ptr,
+                                    const int32_t* seg_start, const int32_t* seg_len, int32_t k,
+                                    void* q, void* k_, const void* v, void* o, void* workspace,
+                                    void* host_workspace, size_t workspace_bytes,
+                                    int32_t* device_status, void* stream) {
+  int st = pp::check_params(params);
+  if (st != PP_OK) return st;
+  const int flags = params->flags;
+  const bool do_rope = !(flags & PP_FLAG_SKIP_ROPE);
+  const bool do_attn = !(flags & PP_FLAG_ROPE_ONLY);
+  if (!q || !k_ || !workspace || !host_workspace) return PP_ERR_INVALID_ARG;
+  if (do_attn && (!v || !o)) return PP_ERR_INVALID_ARG;
+  st = pp::validate_packing(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k);
+  if (st != PP_OK) return st;
+  if (!pp::aligned16(q) || !pp::aligned16(k_) || !pp::aligned16(workspace) ||
+      (do_attn && (!pp::aligned16(v) || !pp::aligned16(o))))
+    return PP_ERR_ALIGNMENT;
+  const size_t need = pp_prefill_workspace_bytes(params, k);
+  if (workspace_bytes < need) return PP_ERR_BUFFER_TOO_SMALL;
+  if ((st = pp::check_device()) != PP_OK) return st;
+
+  pp::TableLayout L;
+  st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
+                                static_cast<int32_t*>(host_workspace), workspace_bytes / sizeof(int32_t), &L);
+  if (st != PP_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * (size_t)L.total_ints,
+                                  cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
+  const int32_t* d_table = static_cast<const int32_t*>(workspace);
+  if (do_rope) {
+    st = pp::launch_rope(*params, d_table, L, q, k_, stream);
+    if (st != PP_OK) return st;
+  }
+  if (do_attn) {
+    st = pp::launch_attention(*params, d_table, L, q, k_, v, o, device_status, stream);
+    if (st != PP_OK) return st;
+  }
+  return PP_OK;
+}
+
+extern "C" size_t pp_unpack_workspace_bytes(int32_t k) { return pp::unpack_table_bytes(k); }
+
+extern "C" int pp_unpack_kv(const pp_attn_params* params, const int32_t* bin_of, const int32_t* off_of,
+                            const int32_t* lengths, int32_t k, const void* k_rot, const void* v,
+                            void* k_cache, void* v_cache, const int64_t* cache_off,
+                            const int32_t* cache_cap, void* workspace, void* host_workspace,
+                            size_t workspace_bytes, void* stream) {
+  int st = pp::check_params(params);
+  if (st != PP_OK) return st;
+  if (!bin_of || !off_of || !lengths || k < 1 || !k_rot || !v || !k_cache || !v_cache || !cache_off ||
+      !cache_cap || !workspace || !host_workspace)
+    return PP_ERR_INVALID_ARG;
+  if (!pp::aligned16(k_rot) || !pp::aligned16(v) || !pp::aligned16(k_cache) || !pp::aligned16(v_cache) ||
+      !pp::aligned16(workspace))
+    return PP_ERR_ALIGNMENT;
+  if (workspace_bytes < pp::unpack_table_bytes(k)) return PP_ERR_BUFFER_TOO_SMALL;
+  int64_t total = 0;
+  for (int32_t i = 0; i < k; ++i) {
+    if (lengths[i] < 1 || cache_cap[i] < lengths[i]) return PP_ERR_LENGTH;
+    if (bin_of[i] < 0 || bin_of[i] >= params->n_bins || off_of[i] < 0 ||
+        (int64_t)off_of[i] + lengths[i] > params->capacity)
+      return PP_ERR_INVALID_ARG;
+    if (cache_off[i] < 0) return PP_ERR_INVALID_ARG;
+    if (cache_off[i] % 8 != 0) return PP_ERR_ALIGNMENT;
+    total += lengths[i];
+    if (total > INT32_MAX) return PP_ERR_UNSUPPORTED;
+  }
+  if ((st = pp::check_device()) != PP_OK) return st;
+
+  auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
+  int32_t* t = static_cast<int32_t*>(host_workspace);
+  std::memset(t, 0, 16);
+  t[0] = k;
+  int32_t* prefix = t + 4;
+  int32_t* h_bin = prefix + up4(k + 1);
+  int32_t* h_off = h_bin + up4(k);
+  int32_t* h_cap = h_off + up4(k);
+  int64_t* h_coff = reinterpret_cast<int64_t*>(h_cap + up4(k));
+  prefix[0] = 0;
+  for (int32_t i = 0; i < k; ++i) {
+    prefix[i + 1] = prefix[i] + lengths[i];
+    h_bin[i] = bin_of[i];
+    h_off[i] = off_of[i];
+    h_cap[i] = cache_cap[i];
+    h_coff[i] = cache_off[i];
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, pp::unpack_table_bytes(k),
+                                  cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "unpack table upload");
+  return pp::launch_unpack(*params, static_cast<const int32_t*>(workspace), k, total, k_rot, v, k_cache,
+                           v_cache, stream);
+}
+
+// ------------------------------------------------------------------------------------------
+// Whole path from host buffers
+// ------------------------------------------------------------------------------------------
+namespace pp {
+namespace {
+
+size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
+
+struct ArenaPlan {
+  size_t q, k, v, o, kc, vc, ws_attn, ws_unpack, status, total;
+};
+
+ArenaPlan plan_arena(const pp_attn_params& p, int32_t n_bins, int32_t capacity, int64_t total_tokens, int32_t k) {
+  ArenaPlan a{};
+  const size_t rows = (size_t)n_bins * capacity;
+  const size_t qb = rows * p.n_q_heads * p.head_dim * 2, kb = rows * p.n_kv_heads * p.head_dim * 2;
+  const size_t cb = (size_t)total_tokens * p.n_kv_heads * p.head_dim * 2;
+  size_t off = 0;
+  a.q = off; off += up256(qb);
+  a.k = off; off += up256(kb);
+  a.v = off; off += up256(kb);
+  a.o = off; off += up256(qb);
+  a.kc = off; off += up256(cb);
+  a.vc = off; off += up256(cb);
+  a.ws_attn = off; off += up256(sizeof(int32_t) * prefill_table_ints(n_bins, capacity, k));
+  a.ws_unpack = off; off += up256(unpack_table_bytes(k));
+  a.status = off; off += 256;
+  a.total = off;
+  return a;
+}
+
+}  // namespace
+}  // namespace pp
+
+extern "C" size_t pp_prefill_host_arena_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k) {
+  if (!params || !lengths || k < 1) return 0;
+  if (params->head_dim != 64 && params->head_dim != 128) return 0;
+  int32_t r = 0, cap = 0;
+  if (pp_pack(lengths, k, 0, &r, &cap, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr) != PP_OK) return 0;
+  int64_t total = 0;
+  for (int32_t i = 0; i < k; ++i) total += lengths[i];
+  return pp::plan_arena(*params, r, cap, total, k).total;
+}
+
+extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, int32_t k,
+                               const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                               void* k_cache_host, void* v_cache_host, void* arena, size_t arena_bytes,
+                               void* stream) {
+  if (!params || !lengths || k < 1 || !q_host || !k_host || !v_host || !o_host || !k_cache_host ||
+      !v_cache_host || !arena)
+    return PP_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(arena) & 255u) return PP_ERR_ALIGNMENT;
+  try {
+    std::vector<int32_t> bin_seg_ptr(k + 1), seg_prompt(k), seg_start(k), seg_len(k), bin_of(k), off_of(k);
+    int32_t r = 0, cap = 0;
+    int st = pp_pack(lengths, k, 0, &r, &cap, bin_seg_ptr.data(), seg_prompt.data(), seg_start.data(),
+                     seg_len.data(), bin_of.data(), off_of.data());
+    if (st != PP_OK) return st;
+    params->capacity = cap;
+    params->n_bins = r;
+    params->flags = 0;
+    if ((st = pp::check_params(params)) != PP_OK) return st;
+    int64_t total = 0;
+    std::vector<int64_t> tok_off(k), cache_off(k);
+    for (int32_t i = 0; i < k; ++i) {
+      tok_off[i] = total;
+      cache_off[i] = total * params->n_kv_heads * params->head_dim;
+      total += lengths[i];
+    }
+    const pp::ArenaPlan a = pp::plan_arena(*params, r, cap, total, k);
+    if (arena_bytes < a.total) return PP_ERR_BUFFER_TOO_SMALL;
+    char* base = static_cast<char*>(arena);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t q_row = (size_t)params->n_q_heads * params->head_dim * 2;
+    const size_t kv_row = (size_t)params->n_kv_heads * params->head_dim * 2;
+    cudaError_t e;
+#define PP_TRY(call, what) do { e = (call); if (e != cudaSuccess) return pp::note_cuda_error((int)e, what); } while (0)
+    // TENSORIZE: zero the packed buffers (padding rows must be finite), then one copy per prompt
+    PP_TRY(cudaMemsetAsync(base + a.q, 0, a.o - a.q, s), "memset packed q/k/v");
+    PP_TRY(cudaMemsetAsync(base + a.status, 0, 4, s), "memset status");
+    for (int32_t i = 0; i < k; ++i) {
+      const size_t row = (size_t)bin_of[i] * cap + off_of[i];
+      PP_TRY(cudaMemcpyAsync(base + a.q + row * q_row, (const char*)q_host + tok_off[i] * q_row,
+                             lengths[i] * q_row, cudaMemcpyHostToDevice, s), "H2D q");
+      PP_TRY(cudaMemcpyAsync(base + a.k + row * kv_row, (const char*)k_host + tok_off[i] * kv_row,
+                             lengths[i] * kv_row, cudaMemcpyHostToDevice, s), "H2D k");
+      PP_TRY(cudaMemcpyAsync(base + a.v + row * kv_row, (const char*)v_host + tok_off[i] * kv_row,
+                             lengths[i] * kv_row, cudaMemcpyHostToDevice, s), "H2D v");
+    }
+    // host staging for the two tables (pageable: the copies below stage them before returning)
+    std::vector<int32_t> h_ws_attn(pp::prefill_table_ints(r, cap, k));
+    std::vector<int64_t> h_ws_unpack((pp::unpack_table_bytes(k) + 7) / 8);
+    st = pp_prefill_attention(params, bin_seg_ptr.data(), seg_start.data(), seg_len.data(), k, base + a.q,
+                              base + a.k, base + a.v, base + a.o, base + a.ws_attn, h_ws_attn.data(),
+                              h_ws_attn.size() * sizeof(int32_t),
+                              reinterpret_cast<int32_t*>(base + a.status), stream);
+    if (st != PP_OK) return st;
+    st = pp_unpack_kv(params, bin_of.data(), off_of.data(), lengths, k, base + a.k, base + a.v, base + a.kc,
+                      base + a.vc, cache_off.data(), lengths, base + a.ws_unpack, h_ws_unpack.data(),
+                      h_ws_unpack.size() * 8, stream);
+    if (st != PP_OK) return st;
+    // UNPACK to the host: caches are already in original order; O goes back prompt by prompt
+    const size_t cache_bytes = (size_t)total * kv_row;
+    PP_TRY(cudaMemcpyAsync(k_cache_host, base + a.kc, cache_bytes, cudaMemcpyDeviceToHost, s), "D2H k cache");
+    PP_TRY(cudaMemcpyAsync(v_cache_host, base + a.vc, cache_bytes, cudaMemcpyDeviceToHost, s), "D2H v cache");
+    for (int32_t i = 0; i < k; ++i) {
+      const size_t row = (size_t)bin_of[i] * cap + off_of[i];
+      PP_TRY(cudaMemcpyAsync((char*)o_host + tok_off[i] * q_row, base + a.o + row * q_row, lengths[i] * q_row,
+                             cudaMemcpyDeviceToHost, s), "D2H o");
+    }
+    int32_t status = 0;
+    PP_TRY(cudaMemcpyAsync(&status, base + a.status, 4, cudaMemcpyDeviceToHost, s), "D2H status");
+    PP_TRY(cudaStreamSynchronize(s), "stream synchronize");
+#undef PP_TRY
+    return status == 0 ? PP_OK : PP_ERR_DEVICE_TIMEOUT;
+  } catch (const std::bad_alloc&) {
+    return PP_ERR_NO_MEMORY;
+  }
+}

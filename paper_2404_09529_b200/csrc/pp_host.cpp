@@ -1,0 +1,230 @@
+// Host side of the prepack-b200 library: BINPACK (first-fit-decreasing), RESTART-PE ids,
+// status strings, and the tile work list that the attention kernel walks.
+// Algorithm 1 lines 2-7 and Sections 3.1-3.2 of the prepacking paper.
+#include "pp_internal.h"
+
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <numeric>
+#include <vector>
+
+extern "C" int pp_version(void) { return 100; }
+
+extern "C" const char* pp_strerror(int status) {
+  switch (status) {
+    case PP_OK: return "ok";
+    case PP_ERR_INVALID_ARG: return "invalid argument";
+    case PP_ERR_LENGTH: return "prompt length < 1 or > bin capacity";
+    case PP_ERR_BUFFER_TOO_SMALL: return "workspace or arena too small";
+    case PP_ERR_UNSUPPORTED: return "unsupported shape or device (needs head_dim 64/128, Hq % Hkv == 0, sm_100)";
+    case PP_ERR_ALIGNMENT: return "device pointer or offset not 16-byte aligned";
+    case PP_ERR_CUDA: return "CUDA call failed";
+    case PP_ERR_DEVICE_TIMEOUT: return "bounded device-side wait gave up";
+    case PP_ERR_NO_MEMORY: return "host allocation failed";
+    default: return "unknown status";
+  }
+}
+
+namespace {
+
+// Tournament tree over bin slots holding each bin's free rows; answers "lowest-numbered bin
+// with at least `need` free rows" in O(log k). Unopened slots hold 0 free rows.
+class FirstFitTree {
+ public:
+  explicit FirstFitTree(int n) {
+    size_ = 1;
+    while (size_ < n) size_ <<= 1;
+    free_.assign(2 * size_, 0);
+  }
+  // Lowest slot index with free >= need, or -1.
+  int find(int need) const {
+    if (free_[1] < need) return -1;
+    int node = 1;
+    while (node < size_) node = (free_[2 * node] >= need) ? 2 * node : 2 * node + 1;
+    return node - size_;
+  }
+  void set(int slot, int value) {
+    int node = slot + size_;
+    free_[node] = value;
+    for (node >>= 1; node >= 1; node >>= 1) free_[node] = std::max(free_[2 * node], free_[2 * node + 1]);
+  }
+  int get(int slot) const { return free_[slot + size_]; }
+
+ private:
+  int size_;
+  std::vector<int> free_;
+};
+
+}  // namespace
+
+extern "C" int pp_pack(const int32_t* lengths, int32_t k, int32_t capacity, int32_t* n_bins,
+                       int32_t* capacity_out, int32_t* bin_seg_ptr, int32_t* seg_prompt,
+                       int32_t* seg_start, int32_t* seg_len, int32_t* bin_of, int32_t* off_of) {
+  if (lengths == nullptr || n_bins == nullptr || k < 1 || capacity < 0) return PP_ERR_INVALID_ARG;
+  int32_t longest = 0;
+  for (int32_t i = 0; i < k; ++i) {
+    if (lengths[i] < 1) return PP_ERR_LENGTH;
+    longest = std::max(longest, lengths[i]);
+  }
+  const int32_t cap = capacity == 0 ? longest : capacity;
+  if (longest > cap) return PP_ERR_LENGTH;
+  try {
+    std::vector<int32_t> order(k);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t a, int32_t b) { return lengths[a] > lengths[b]; });
+    FirstFitTree tree(k);
+    std::vector<int32_t> item_bin(k), item_off(k), bin_count;
+    int32_t r = 0;
+    for (int32_t idx = 0; idx < k; ++idx) {
+      const int32_t i = order[idx];
+      int b = tree.find(lengths[i]);
+      if (b < 0) {            // open a new bin
+        b = r++;
+        tree.set(b, cap);
+        bin_count.push_back(0);
+      }
+      const int32_t free_rows = tree.get(b);
+      item_bin[i] = b;
+      item_off[i] = cap - free_rows;
+      tree.set(b, free_rows - lengths[i]);
+      bin_count[b] += 1;
+    }
+    // CSR over segments, bin-major, placement order inside a bin (= the order items were taken)
+    std::vector<int32_t> ptr(r + 1, 0);
+    for (int32_t b = 0; b < r; ++b) ptr[b + 1] = ptr[b] + bin_count[b];
+    std::vector<int32_t> cursor(ptr.begin(), ptr.end() - 1);
+    for (int32_t idx = 0; idx < k; ++idx) {
+      const int32_t i = order[idx];
+      const int32_t s = cursor[item_bin[i]]++;
+      if (seg_prompt) seg_prompt[s] = i;
+      if (seg_start) seg_start[s] = item_off[i];
+      if (seg_len) seg_len[s] = lengths[i];
+    }
+    if (bin_seg_ptr) std::copy(ptr.begin(), ptr.end(), bin_seg_ptr);
+    if (bin_of) std::copy(item_bin.begin(), item_bin.end(), bin_of);
+    if (off_of) std::copy(item_off.begin(), item_off.end(), off_of);
+    *n_bins = r;
+    if (capacity_out) *capacity_out = cap;
+  } catch (const std::bad_alloc&) {
+    return PP_ERR_NO_MEMORY;
+  }
+  return PP_OK;
+}
+
+namespace pp {
+
+int validate_packing(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
+                     const int32_t* seg_start, const int32_t* seg_len, int32_t k) {
+  if (!bin_seg_ptr || !seg_start || !seg_len || n_bins < 1 || capacity < 1 || k < 1)
+    return PP_ERR_INVALID_ARG;
+  if (bin_seg_ptr[0] != 0 || bin_seg_ptr[n_bins] != k) return PP_ERR_INVALID_ARG;
+  for (int32_t b = 0; b < n_bins; ++b) {
+    if (bin_seg_ptr[b + 1] <= bin_seg_ptr[b]) return PP_ERR_INVALID_ARG;   // no empty bins
+    int64_t off = 0;
+    for (int32_t s = bin_seg_ptr[b]; s < bin_seg_ptr[b + 1]; ++s) {
+      if (seg_len[s] < 1) return PP_ERR_LENGTH;
+      if (seg_start[s] != off) return PP_ERR_INVALID_ARG;                  // contiguous from row 0
+      off += seg_len[s];
+      if (off > capacity) return PP_ERR_LENGTH;
+    }
+  }
+  return PP_OK;
+}
+
+}  // namespace pp
+
+extern "C" int pp_fill_position_ids(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
+                                    const int32_t* seg_start, const int32_t* seg_len,
+                                    int32_t* position_ids, int32_t* segment_ids) {
+  if (!bin_seg_ptr || n_bins < 1) return PP_ERR_INVALID_ARG;
+  const int32_t k = bin_seg_ptr[n_bins];
+  const int st = pp::validate_packing(n_bins, capacity, bin_seg_ptr, seg_start, seg_len, k);
+  if (st != PP_OK) return st;
+  for (int32_t b = 0; b < n_bins; ++b) {
+    int32_t* pos = position_ids ? position_ids + (size_t)b * capacity : nullptr;
+    int32_t* sid = segment_ids ? segment_ids + (size_t)b * capacity : nullptr;
+    int32_t row = 0;
+    for (int32_t s = bin_seg_ptr[b]; s < bin_seg_ptr[b + 1]; ++s)
+      for (int32_t p = 0; p < seg_len[s]; ++p, ++row) {
+        if (pos) pos[row] = p;
+        if (sid) sid[row] = s;
+      }
+    for (; row < capacity; ++row) {
+      if (pos) pos[row] = 0;
+      if (sid) sid[row] = -1;
+    }
+  }
+  return PP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Tile work list (Section 3.2: the independent mask is block lower-triangular per prompt span,
+// so a query tile only ever needs the key rows from the start of the first prompt it touches
+// up to its own last row).
+// ------------------------------------------------------------------------------------------
+namespace pp {
+
+size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k) {
+  const int64_t q_tiles = (int64_t)n_bins * ((capacity + kTileM - 1) / kTileM);
+  // header + bin_seg_ptr + bin_used + seg_start + items (4 ints each), each block 4-int aligned
+  auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
+  return (size_t)(kHeaderInts + up4(n_bins + 1) + up4(n_bins) + up4(k) + 4 * q_tiles);
+}
+
+int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
+                         const int32_t* seg_start, const int32_t* seg_len, int32_t k,
+                         int32_t* out, size_t out_ints, TableLayout* layout) {
+  auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
+  TableLayout L;
+  L.bin_seg_ptr = kHeaderInts;
+  L.bin_used = L.bin_seg_ptr + (int32_t)up4(n_bins + 1);
+  L.seg_start = L.bin_used + (int32_t)up4(n_bins);
+  L.items = L.seg_start + (int32_t)up4(k);
+  if (out_ints < prefill_table_ints(n_bins, capacity, k)) return PP_ERR_BUFFER_TOO_SMALL;
+  std::memset(out, 0, sizeof(int32_t) * (size_t)L.items);
+  std::memcpy(out + L.bin_seg_ptr, bin_seg_ptr, sizeof(int32_t) * (size_t)(n_bins + 1));
+  std::memcpy(out + L.seg_start, seg_start, sizeof(int32_t) * (size_t)k);
+  struct Item { int32_t bin, q_row0, kv_row0, n_kv_tiles; };
+  std::vector<Item> items;
+  try {
+    for (int32_t b = 0; b < n_bins; ++b) {
+      const int32_t s_lo = bin_seg_ptr[b], s_hi = bin_seg_ptr[b + 1];
+      const int32_t used = seg_start[s_hi - 1] + seg_len[s_hi - 1];
+      out[L.bin_used + b] = used;
+      int32_t s = s_lo;
+      for (int32_t q0 = 0; q0 < used; q0 += kTileM) {
+        while (s + 1 < s_hi && seg_start[s + 1] <= q0) ++s;       // segment holding row q0
+        const int32_t kv_lo = (seg_start[s] / kTileN) * kTileN;
+        const int32_t kv_end = std::min(q0 + kTileM, used);
+        items.push_back({b, q0, kv_lo, (kv_end - kv_lo + kTileN - 1) / kTileN});
+      }
+    }
+    // Longest first so that the hardware block scheduler, which hands out blocks in index
+    // order, does longest-processing-time-first scheduling; ties keep bin/row order.
+    std::stable_sort(items.begin(), items.end(),
+                     [](const Item& a, const Item& b) { return a.n_kv_tiles > b.n_kv_tiles; });
+  } catch (const std::bad_alloc&) {
+    return PP_ERR_NO_MEMORY;
+  }
+  std::memcpy(out + L.items, items.data(), sizeof(Item) * items.size());
+  L.n_items = (int32_t)items.size();
+  out[0] = 0x50504b31;  // "PPK1"
+  out[1] = L.n_items;
+  out[2] = n_bins;
+  out[3] = capacity;
+  out[4] = k;
+  out[5] = L.bin_seg_ptr;
+  out[6] = L.bin_used;
+  out[7] = L.seg_start;
+  out[8] = L.items;
+  int64_t tiles = 0;
+  for (const Item& it : items) tiles += it.n_kv_tiles;
+  out[9] = (int32_t)std::min<int64_t>(tiles, INT32_MAX);
+  L.total_ints = (int32_t)(L.items + 4 * (int64_t)items.size());
+  if (layout) *layout = L;
+  return PP_OK;
+}
+
+}  // namespace pp

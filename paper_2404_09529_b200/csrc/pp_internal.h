@@ -1,0 +1,52 @@
+// Internal declarations shared by the translation units of the prepack-b200 library.
+#ifndef PREPACK_B200_PP_INTERNAL_H_
+#define PREPACK_B200_PP_INTERNAL_H_
+
+#include <cstddef>
+#include <cstdint>
+
+#include "../../include/pp.h"
+
+namespace pp {
+
+constexpr int kTileM = 128;      // query rows per work item (tcgen05 MMA M)
+constexpr int kTileN = 128;      // key rows per inner step (tcgen05 MMA N of Q.K^T)
+constexpr int kHeaderInts = 16;  // table header, see build_prefill_tables
+
+// Offsets (in int32 units) of the blocks inside the prefill table that is built on the host and
+// copied to the device workspace.
+struct TableLayout {
+  int32_t bin_seg_ptr = 0;  // [R+1]
+  int32_t bin_used = 0;     // [R]   occupied rows per bin
+  int32_t seg_start = 0;    // [k]   bin-local first row of each segment
+  int32_t items = 0;        // [n_items][4] = (bin, q_row0, kv_row0, n_kv_tiles), longest first
+  int32_t n_items = 0;
+  int32_t total_ints = 0;
+};
+
+int validate_packing(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
+                     const int32_t* seg_start, const int32_t* seg_len, int32_t k);
+size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k);
+int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
+                         const int32_t* seg_start, const int32_t* seg_len, int32_t k,
+                         int32_t* out, size_t out_ints, TableLayout* layout);
+
+// Records a failed CUDA call for pp_last_cuda_error(); returns PP_ERR_CUDA.
+int note_cuda_error(int cuda_error, const char* what);
+
+// Kernel launchers (device pointers, stream = cudaStream_t as void*). Return a PP_* status.
+int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
+                void* q, void* k, void* stream);
+int launch_attention(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
+                     const void* q, const void* k, const void* v, void* o,
+                     int32_t* device_status, void* stream);
+int launch_unpack(const pp_attn_params& p, const int32_t* d_table, int32_t k, int64_t total_tokens,
+                  const void* k_rot, const void* v, void* k_cache, void* v_cache, void* stream);
+
+// Unpack table (int32 units): header 4 ints, then token_prefix[k+1], bin_of[k], off_of[k],
+// cache_cap[k], cache_off as int64[k] (8-byte aligned).
+size_t unpack_table_bytes(int32_t k);
+
+}  // namespace pp
+
+#endif  // PREPACK_B200_PP_INTERNAL_H_

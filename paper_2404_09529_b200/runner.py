@@ -1,0 +1,112 @@
+"""Memory plumbing around the C-ABI calls: lays token-major tensors out as the packed (or padded)
+batch, owns the device buffers and workspaces, and calls pp_pack / pp_prefill_attention /
+pp_unpack_kv in order. All arithmetic of the method happens inside the library."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class PrefillBatch:
+    """One batch of prompts on the device, ready to be prefilled.
+
+    mode "packed": bins from pp_pack(lengths) (first-fit-decreasing, capacity = longest prompt).
+    mode "padded": the full-batching baseline -- one bin per prompt in original order, every
+    bin declared as a single segment of the full capacity, so all k*m rows are computed;
+    unpack still copies only each prompt's true rows.
+    """
+
+    def __init__(self, lengths, n_q_heads: int, n_kv_heads: int, head_dim: int, rope_base: float,
+                 mode: str = "packed", device: str = "cuda", softmax_scale: float = 0.0):
+        self.device = torch.device(device)
+        self.mode = mode
+        self.lengths = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
+        self.k = int(self.lengths.shape[0])
+        self.total_tokens = int(self.lengths.sum())
+        self.hq, self.hkv, self.d = n_q_heads, n_kv_heads, head_dim
+        self.rope_base, self.softmax_scale = rope_base, softmax_scale
+        self._pack()
+        R, M = self.pack.n_bins, self.pack.capacity
+        dev, bf = self.device, torch.bfloat16
+        self.q = torch.zeros((R, M, n_q_heads, head_dim), dtype=bf, device=dev)
+        self.kk = torch.zeros((R, M, n_kv_heads, head_dim), dtype=bf, device=dev)
+        self.v = torch.zeros((R, M, n_kv_heads, head_dim), dtype=bf, device=dev)
+        self.o = torch.zeros((R, M, n_q_heads, head_dim), dtype=bf, device=dev)
+        # per-prompt caches, one pool each, [Hkv, l_i, D] blocks back to back in original order
+        self.cache_cap = self.lengths.copy()
+        tok_prefix = np.concatenate([[0], np.cumsum(self.lengths.astype(np.int64))])
+        self.cache_off = (tok_prefix[:-1] * n_kv_heads * head_dim).astype(np.int64)
+        pool = self.total_tokens * n_kv_heads * head_dim
+        self.k_cache = torch.zeros(pool, dtype=bf, device=dev)
+        self.v_cache = torch.zeros(pool, dtype=bf, device=dev)
+        self.ws = B.Workspaces(self.params, self.pack.k, device=dev)
+        # flat packed row of every real token, original prompt order
+        rows = [np.arange(l, dtype=np.int64) + int(b) * M + int(off)
+                for l, b, off in zip(self.lengths, self.bin_of, self.off_of)]
+        self.token_rows = torch.from_numpy(np.concatenate(rows)).to(dev)
+
+    def _pack(self) -> None:
+        """BINPACK through the library (host)."""
+        if self.mode == "packed":
+            self.pack = B.pp_pack(self.lengths, 0)
+            self.bin_of, self.off_of = self.pack.bin_of, self.pack.off_of
+        elif self.mode == "padded":
+            m = int(self.lengths.max())
+            self.pack = B.pp_pack(np.full(self.k, m, dtype=np.int32), 0)
+            self.bin_of = np.arange(self.k, dtype=np.int32)
+            self.off_of = np.zeros(self.k, dtype=np.int32)
+        else:
+            raise ValueError(self.mode)
+        self.params = B.AttnParams(self.hq, self.hkv, self.d, self.rope_base, self.softmax_scale,
+                                   self.pack.capacity, self.pack.n_bins, 0)
+
+    def load(self, q_tok: torch.Tensor, k_tok: torch.Tensor, v_tok: torch.Tensor) -> None:
+        """TENSORIZE: scatter token-major [T, H, D] tensors into the packed layout; padding rows zero."""
+        for dst, src in ((self.q, q_tok), (self.kk, k_tok), (self.v, v_tok)):
+            dst.zero_()
+            dst.view(-1, dst.shape[2], dst.shape[3])[self.token_rows] = src.to(self.device)
+
+    def run(self, flags: int = 0, repack: bool = False, unpack: bool = True) -> None:
+        """One pass of the hot path on the current stream (asynchronous)."""
+        if repack:
+            self._pack()
+        stream = torch.cuda.current_stream().cuda_stream
+        host_attn, host_unpack, slot = self.ws.acquire()
+        self.params.flags = flags
+        B.pp_prefill_attention(self.params, self.pack, self.q, self.kk, self.v, self.o, self.ws.attn_dev,
+                               host_attn, self.ws.attn_bytes, self.ws.status, stream)
+        if unpack:
+            B.pp_unpack_kv(self.params, self.bin_of, self.off_of, self.lengths, self.kk, self.v, self.k_cache,
+                           self.v_cache, self.cache_off, self.cache_cap, self.ws.unpack_dev, host_unpack,
+                           self.ws.unpack_bytes, stream)
+        self.ws.release(slot)
+
+    def run_unpack_only(self) -> None:
+        stream = torch.cuda.current_stream().cuda_stream
+        _, host_unpack, slot = self.ws.acquire()
+        B.pp_unpack_kv(self.params, self.bin_of, self.off_of, self.lengths, self.kk, self.v, self.k_cache,
+                       self.v_cache, self.cache_off, self.cache_cap, self.ws.unpack_dev, host_unpack,
+                       self.ws.unpack_bytes, stream)
+        self.ws.release(slot)
+
+    def device_status(self) -> int:
+        return int(self.ws.status.item())
+
+    # ---- views of the results, original prompt order (device tensors) ----
+    def o_tokens(self) -> torch.Tensor:
+        """[T, Hq, D] attention outputs of the real tokens."""
+        return self.o.view(-1, self.hq, self.d)[self.token_rows]
+
+    def rotated_tokens(self):
+        """([T, Hq, D], [T, Hkv, D]): q and k as they stand in the packed buffers."""
+        return (self.q.view(-1, self.hq, self.d)[self.token_rows],
+                self.kk.view(-1, self.hkv, self.d)[self.token_rows])
+
+    def caches(self, i: int):
+        """(k_cache_i, v_cache_i) as [Hkv, l_i, D] views of the pools."""
+        n = int(self.lengths[i]) * self.hkv * self.d
+        off = int(self.cache_off[i])
+        shape = (self.hkv, int(self.cache_cap[i]), self.d)
+        return self.k_cache[off:off + n].view(shape), self.v_cache[off:off + n].view(shape)

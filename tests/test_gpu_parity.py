@@ -1,0 +1,162 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the float64 oracle.
+Tolerances are the spec ones (max-abs 2e-2, mean-abs 2e-3 for bf16 outputs and caches);
+V caches, packing indices and everything that is a pure copy must match bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from parity_utils import compare_full, compare_sampled, run_cuda, to64
+from workloads import CONFIGS, make_qkv, prompt_lengths, split_by_prompt
+
+pytestmark = pytest.mark.gpu
+
+
+def _workload(name, device="cpu"):
+    cfg = CONFIGS[name]
+    lengths = prompt_lengths(name)
+    q, k, v = make_qkv(cfg, int(lengths.sum()), device=device)
+    return cfg, lengths, q, k, v
+
+
+def _random_case(lengths, hq, hkv, d, seed):
+    g = torch.Generator().manual_seed(seed)
+    t = int(np.sum(lengths))
+    mk = lambda h: torch.randn((t, h, d), generator=g).to(torch.bfloat16)
+    return mk(hq), mk(hkv), mk(hkv)
+
+
+@pytest.mark.parametrize("mode", ["packed", "padded"])
+def test_tiny_full_parity(mode):
+    cfg, lengths, q, k, v = _workload("tiny")
+    batch = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, mode)
+    compare_full(batch, lengths, q, k, v, cfg.rope_base)
+    # RoPE at position 0 is the identity; the first token attends only to itself
+    ks, vs = split_by_prompt(k, lengths), split_by_prompt(v, lengths)
+    os_ = split_by_prompt(batch.o_tokens().cpu(), lengths)
+    for i in range(len(lengths)):
+        kc, vc = batch.caches(i)
+        assert torch.equal(kc[:, 0, :].cpu(), ks[i][0])
+        assert torch.equal(os_[i][0], vs[i][0])           # MHA: head h reads KV head h
+
+
+def test_packed_and_padded_caches_are_bit_identical():
+    cfg, lengths, q, k, v = _workload("tiny")
+    a = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, "packed")
+    b = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, "padded")
+    assert torch.equal(a.k_cache, b.k_cache) and torch.equal(a.v_cache, b.v_cache)
+    assert float((a.o_tokens().float() - b.o_tokens().float()).abs().max()) <= 2e-2
+
+
+def test_llama2_7b_full_parity_packed():
+    cfg, lengths, q, k, v = _workload("llama2_7b")
+    batch = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    # every cache element and every O row of 12 prompts (longest, shortest and ten others)
+    order = np.argsort(lengths)
+    prompts = sorted(set([int(order[0]), int(order[-1])] + [int(x) for x in order[3::6]]))
+    compare_full(batch, lengths, q, k, v, cfg.rope_base, prompts=prompts)
+
+
+def test_llama2_7b_sampled_parity_padded():
+    cfg, lengths, q, k, v = _workload("llama2_7b")
+    batch = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, "padded")
+    compare_sampled(batch, lengths, q, k, v, cfg.rope_base, prompts=list(range(0, 64, 5)),
+                    kv_heads=[0, 17, 31], n_rows=48)
+
+
+def test_many_short_full_parity_packed():
+    cfg, lengths, q, k, v = _workload("many_short")
+    batch = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    order = np.argsort(lengths)
+    prompts = sorted(set([int(x) for x in order[-6:]] + [int(x) for x in order[::37]]))
+    compare_full(batch, lengths, q, k, v, cfg.rope_base, prompts=prompts)
+
+
+@pytest.mark.parametrize("name", ["llama3_8b_gqa", "long_mix"])
+def test_large_configs_sampled_parity_packed(name):
+    """Full-size launch, sampled outputs: a few prompts (longest, shortest, some in between), the
+    query heads of two KV heads, ~40 query rows each, and those KV heads' whole caches."""
+    cfg, lengths, q, k, v = _workload(name, device="cuda")
+    batch = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    order = np.argsort(lengths)
+    prompts = sorted(set(int(order[i]) for i in (0, 1, len(order) // 2, -3, -1)))
+    compare_sampled(batch, lengths, q.cpu(), k.cpu(), v.cpu(), cfg.rope_base, prompts=prompts,
+                    kv_heads=[1, cfg.n_kv_heads - 1], n_rows=40)
+
+
+@pytest.mark.parametrize("lengths,hq,hkv,d", [
+    ([1], 2, 2, 64),                       # a single one-token prompt
+    ([128], 4, 1, 128),                    # exactly one tile, GQA group 4
+    ([128, 128, 128], 2, 2, 128),          # tile-aligned prompts, worst case r = k
+    ([129, 1, 1, 127], 2, 1, 64),          # ragged tails and one-token prompts sharing bins
+    ([700, 300, 250, 150, 90, 5, 5], 8, 2, 128),   # several tiles, segments straddling tiles
+    ([515, 130, 129, 128, 64, 33, 17, 9, 3, 2, 1], 8, 1, 64),   # group 8, D = 64
+    ([8] * 40, 2, 2, 64),                  # many equal short prompts: 16 segments per tile
+])
+def test_edge_shapes_full_parity(lengths, hq, hkv, d):
+    q, k, v = _random_case(lengths, hq, hkv, d, seed=len(lengths) * 1000 + d)
+    for mode in ("packed", "padded"):
+        batch = run_cuda(lengths, q, k, v, hq, hkv, d, 10000.0, mode)
+        compare_full(batch, np.asarray(lengths), q, k, v, 10000.0)
+
+
+def test_no_cross_prompt_attention_on_gpu():
+    """Overwrite one prompt with large finite values: every other prompt's output and caches
+    stay bit-identical (Section 3.2, independent masking)."""
+    cfg, lengths, q, k, v = _workload("tiny")
+    a = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    victim = 6                                  # shares bin 1 with prompt 1, placed after it
+    prefix = np.concatenate([[0], np.cumsum(lengths)])
+    q2, k2, v2 = q.clone(), k.clone(), v.clone()
+    sl = slice(int(prefix[victim]), int(prefix[victim + 1]))
+    q2[sl] = 3000.0; k2[sl] = -2500.0; v2[sl] = 1.0e4
+    b = run_cuda(lengths, q2, k2, v2, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    oa, ob = split_by_prompt(a.o_tokens().cpu(), lengths), split_by_prompt(b.o_tokens().cpu(), lengths)
+    for i in range(len(lengths)):
+        if i == victim:
+            continue
+        assert torch.equal(oa[i], ob[i]), i
+        assert torch.equal(a.caches(i)[0], b.caches(i)[0]) and torch.equal(a.caches(i)[1], b.caches(i)[1])
+    # same for a prompt placed before its bin mates
+    victim = 2
+    q2, k2, v2 = q.clone(), k.clone(), v.clone()
+    sl = slice(int(prefix[victim]), int(prefix[victim + 1]))
+    q2[sl] = -3000.0; k2[sl] = 2500.0; v2[sl] = -1.0e4
+    b = run_cuda(lengths, q2, k2, v2, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    ob = split_by_prompt(b.o_tokens().cpu(), lengths)
+    for i in range(len(lengths)):
+        if i != victim:
+            assert torch.equal(oa[i], ob[i]), i
+
+
+def test_explicit_capacity_and_skip_rope_flags():
+    import paper_2404_09529_b200 as pp
+    from paper_2404_09529_b200.runner import PrefillBatch
+    lengths = np.array([200, 77, 130, 31], np.int32)
+    q, k, v = _random_case(lengths, 4, 2, 128, seed=5)
+    ref = run_cuda(lengths, q, k, v, 4, 2, 128, 500000.0)
+    # rope-only then attention-only gives the same bits as the fused call
+    b = PrefillBatch(lengths, 4, 2, 128, 500000.0)
+    b.load(q, k, v)
+    b.run(flags=pp.PP_FLAG_ROPE_ONLY, unpack=False)
+    b.run(flags=pp.PP_FLAG_SKIP_ROPE)
+    torch.cuda.synchronize()
+    assert torch.equal(b.o_tokens(), ref.o_tokens())
+    assert torch.equal(b.k_cache, ref.k_cache) and torch.equal(b.v_cache, ref.v_cache)
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    import paper_2404_09529_b200 as pp
+    cfg, lengths, q, k, v = _workload("tiny")
+    ref = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    params = pp.AttnParams(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, 0.0, 0, 0, 0)
+    nbytes = pp.pp_prefill_host_arena_bytes(params, lengths)
+    assert nbytes > 0
+    arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    o = torch.empty_like(q)
+    kc = torch.empty(k.numel(), dtype=torch.bfloat16)
+    vc = torch.empty(v.numel(), dtype=torch.bfloat16)
+    pp.pp_prefill_host(params, lengths, q.contiguous(), k.contiguous(), v.contiguous(), o, kc, vc, arena, nbytes,
+                       torch.cuda.current_stream().cuda_stream)
+    assert (params.n_bins, params.capacity) == (4, 112)
+    assert torch.equal(o, ref.o_tokens().cpu())
+    assert torch.equal(kc, ref.k_cache.cpu()) and torch.equal(vc, ref.v_cache.cpu())
