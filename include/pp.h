@@ -42,7 +42,8 @@ enum {
   PP_ERR_ALIGNMENT = -5,        /* a device tensor pointer is not 16-byte aligned              */
   PP_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed (see pp_last_cuda_error)  */
   PP_ERR_DEVICE_TIMEOUT = -7,   /* a bounded device-side wait gave up (device status word)     */
-  PP_ERR_NO_MEMORY = -8         /* host allocation failed                                      */
+  PP_ERR_NO_MEMORY = -8,        /* host allocation failed                                      */
+  PP_ERR_TOO_LARGE = -9         /* more prompts than the built-in scratch of a *_static call   */
 };
 
 /* Flags for pp_attn_params.flags */
@@ -163,6 +164,28 @@ int pp_unpack_kv(const pp_attn_params* params,
                  const void* k_rot, const void* v, void* k_cache, void* v_cache,
                  const int64_t* cache_off, const int32_t* cache_cap,
                  void* workspace, void* host_workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * pp_unpack_kv without a caller workspace (the paper has no counterpart; this is for users of the
+ * library who may not allocate device memory: a serving process whose pool was carved up at
+ * start-up, a plug-in that receives tensors but no allocator, code running while another
+ * component owns the allocator). Arguments and result are those of pp_unpack_kv minus the two
+ * workspaces: the per-prompt table lives in a fixed device array inside the library image (about
+ * 96 KiB on every GPU that loads the library, held until the process exits), so
+ *   - k may not exceed pp_unpack_static_max_prompts() (4096); more gives PP_ERR_TOO_LARGE and
+ *     nothing is enqueued;
+ *   - the call allocates nothing, on the host or on the device;
+ *   - the first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture;
+ *   - all calls on one GPU share the one table: two calls whose device work can overlap (different
+ *     streams, or different host threads without ordering between their streams) race on it.
+ *     Calls on the same stream are safe, and the table is rewritten in full on every call.
+ */
+int32_t pp_unpack_static_max_prompts(void);
+int pp_unpack_kv_static(const pp_attn_params* params,
+                        const int32_t* bin_of, const int32_t* off_of, const int32_t* lengths, int32_t k,
+                        const void* k_rot, const void* v, void* k_cache, void* v_cache,
+                        const int64_t* cache_off, const int32_t* cache_cap, void* stream);
 
 /*
  * Whole path from host memory (Algorithm 1 lines 2-8 for one attention layer), for callers whose

@@ -8,12 +8,14 @@ from .binding import (PP_FLAG_ROPE_ONLY, PP_FLAG_SKIP_ROPE, AttnParams, Packing,
                       Workspaces, lib_path, load_library, pp_fill_position_ids,
                       pp_last_cuda_error, pp_pack, pp_prefill_attention, pp_prefill_host,
                       pp_prefill_host_arena_bytes, pp_prefill_workspace_bytes, pp_strerror,
-                      pp_unpack_kv, pp_unpack_workspace_bytes, pp_version)
+                      pp_unpack_kv, pp_unpack_kv_static, pp_unpack_static_max_prompts,
+                      pp_unpack_workspace_bytes, pp_version)
 
 __all__ = [
     "PP_FLAG_ROPE_ONLY", "PP_FLAG_SKIP_ROPE", "AttnParams", "Packing", "PrepackError", "Workspaces",
     "lib_path", "load_library", "pp_fill_position_ids", "pp_last_cuda_error", "pp_pack",
     "pp_prefill_attention", "pp_prefill_host", "pp_prefill_host_arena_bytes",
-    "pp_prefill_workspace_bytes", "pp_strerror", "pp_unpack_kv", "pp_unpack_workspace_bytes",
+    "pp_prefill_workspace_bytes", "pp_strerror", "pp_unpack_kv", "pp_unpack_kv_static",
+    "pp_unpack_static_max_prompts", "pp_unpack_workspace_bytes",
     "pp_version",
 ]

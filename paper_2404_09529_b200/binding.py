@@ -60,6 +60,8 @@ def load_library():
         "pp_unpack_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32]),
         "pp_unpack_kv": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, i64p, i32p, vp, vp,
                                         ctypes.c_size_t, vp]),
+        "pp_unpack_static_max_prompts": (ctypes.c_int32, []),
+        "pp_unpack_kv_static": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, i64p, i32p, vp]),
         "pp_prefill_host_arena_bytes": (ctypes.c_size_t, [pp, i32p, ctypes.c_int32]),
         "pp_prefill_host": (ctypes.c_int, [pp, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]),
     }
@@ -174,6 +176,22 @@ def pp_unpack_kv(params: AttnParams, bin_of, off_of, lengths, k_rot, v, k_cache,
         _addr(k_cache), _addr(v_cache), co.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), _p32(cc),
         _addr(workspace), _addr(host_workspace), workspace_bytes, stream)
     _check(st, "pp_unpack_kv")
+
+
+def pp_unpack_static_max_prompts() -> int:
+    return int(load_library().pp_unpack_static_max_prompts())
+
+
+def pp_unpack_kv_static(params: AttnParams, bin_of, off_of, lengths, k_rot, v, k_cache, v_cache, cache_off,
+                        cache_cap, stream: int = 0) -> None:
+    """pp_unpack_kv for callers that cannot allocate: no workspaces, at most
+    pp_unpack_static_max_prompts() prompts, one shared table per GPU (see include/pp.h)."""
+    b, o, l, cc = _i32(bin_of), _i32(off_of), _i32(lengths), _i32(cache_cap)
+    co = np.ascontiguousarray(np.asarray(cache_off, dtype=np.int64))
+    st = load_library().pp_unpack_kv_static(
+        ctypes.byref(params), _p32(b), _p32(o), _p32(l), int(l.shape[0]), _addr(k_rot), _addr(v),
+        _addr(k_cache), _addr(v_cache), co.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), _p32(cc), stream)
+    _check(st, "pp_unpack_kv_static")
 
 
 def pp_prefill_host_arena_bytes(params: AttnParams, lengths) -> int:

@@ -22,6 +22,7 @@ extern "C" const char* pp_strerror(int status) {
     case PP_ERR_CUDA: return "CUDA call failed";
     case PP_ERR_DEVICE_TIMEOUT: return "bounded device-side wait gave up";
     case PP_ERR_NO_MEMORY: return "host allocation failed";
+    case PP_ERR_TOO_LARGE: return "more prompts than the built-in scratch of the static entry point holds";
     default: return "unknown status";
   }
 }
