@@ -81,14 +81,16 @@ extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t*
   if ((st = pp::check_device()) != PP_OK) return st;
 
   pp::TableLayout L;
-  st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
+  // an even number of query heads per KV head pairs two heads per work item, else two row tiles
+  const bool pair_rows = ((params->n_q_heads / params->n_kv_heads) % 2) != 0;
+  st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k, pair_rows,
                                 static_cast<int32_t*>(host_workspace), workspace_bytes / sizeof(int32_t), &L);
   if (st != PP_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * (size_t)L.total_ints,
                                   cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
-  const int32_t* d_table = static_cast<const int32_t*>(workspace);
+  int32_t* d_table = static_cast<int32_t*>(workspace);
   if (do_rope) {
     st = pp::launch_rope(*params, d_table, L, q, k_, stream);
     if (st != PP_OK) return st;

@@ -2,15 +2,22 @@
 //   o_i = sum_j softmax_j(q'_i . k'_j * scale) v_j   over keys j of the same prompt with j <= i.
 // The independent mask M' (a lower-triangular block per prompt span) is never built: every query
 // row carries the key range [start row of its prompt, its own row], and the host work list
-// restricts each 128-row query tile to the key tiles that can intersect such a range.
+// restricts each query tile to the key tiles that can intersect such a range.
 //
-// One CTA = one (query tile, query head). Warp roles:
-//   warp 0      TMA producer (Q once, then the K and V tiles of the key loop), TMEM allocator
-//   warp 1      tcgen05.mma issuer: S = Q K^T into TMEM, then O += P V with P read from TMEM
-//   warps 2-5   online softmax, one query row per thread (TMEM lane = row): tcgen05.ld S,
-//               mask, exp2, tcgen05.st P (bf16, over the S columns), rescale O when the running
-//               maximum moved, and the epilogue (O / l -> bf16 -> shared -> TMA store)
-// Two CTAs share an SM (256 TMEM columns each), so one CTA's MMAs overlap the other's softmax.
+// Persistent kernel, one CTA per SM, 384 threads. Each CTA draws work items from a global counter
+// (items are listed KV-head-major, longest first). A work item has two 128-row query-tile slots
+// that share one stream of 128-row key/value tiles: two query heads of one KV head over the same
+// rows (even GQA group), or two consecutive row tiles of one head.
+//   warp 0       producer: draws items, TMA-loads Q (per slot) and the K / V tile rings
+//   warp 1       issues tcgen05.mma: S_t = Q_t K^T into TMEM, O_t += P_t V with P_t read from TMEM;
+//                the two slots alternate (S0, S1, then PV0, S0', PV1, S1', ...) so that one slot's
+//                MMAs run while the other slot's softmax works
+//   warps 4-7    softmax of slot 0, one query row per thread (TMEM lane = row)
+//   warps 8-11   softmax of slot 1
+// Softmax: tcgen05.ld the 128 scores of the row, mask to the row's key range, lazy running maximum
+// (O is rescaled only when the maximum grows by more than 2^8), exp2, P written as bf16 over the S
+// columns, and at the end of an item O / l is stored straight to global memory.
+// TMEM: S0 | S1 | O0 | O1 = 512 columns. Every mbarrier wait is bounded.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <cuda_bf16.h>
@@ -18,6 +25,7 @@
 
 #include <cmath>
 #include <cstdlib>
+#include <type_traits>
 
 #include "pp_internal.h"
 
@@ -26,19 +34,22 @@ namespace {
 
 constexpr int BM = kTileM;
 constexpr int BN = kTileN;
-constexpr int kAttnThreads = 192;
-constexpr int kSoftmaxThreads = 128;
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kTmemColS = 0;      // S (fp32, BN columns); P (bf16 pairs, BN/2 columns) aliases it
-constexpr uint32_t kTmemColO = 128;    // O (fp32, D columns)
+constexpr int kAttnThreads = 384;
+constexpr int kSoftmaxThreads = 128;       // per slot
+constexpr uint32_t kTmemCols = 512;
+constexpr int kRegsSoftmax = 200;          // setmaxnreg budgets: 128*104 + 256*200 <= 65536
+constexpr int kRegsOther = 104;
 
 template <int D> struct AttnCfg {
-  static constexpr int kStages = (D == 128) ? 1 : 2;
+  static constexpr int kKStages = (D == 128) ? 3 : 4;
+  static constexpr int kVStages = (D == 128) ? 2 : 4;
   static constexpr int kChunks = D / 64;                     // 128-byte swizzle spans per row
-  static constexpr int kQBytes = BM * D * 2;
+  static constexpr int kQBytes = BM * D * 2;                 // per slot
   static constexpr int kKVBytes = BN * D * 2;
-  static constexpr int kBarBytes = 256;
-  static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kQBytes + 2 * kStages * kKVBytes + kBarBytes;
+  static constexpr int kMiscBytes = 512;
+  static constexpr int kSmemBytes = 1024 /*alignment slack*/ + 2 * kQBytes + (kKStages + kVStages) * kKVBytes + kMiscBytes;
+  static constexpr uint32_t kTmemS = 0;                      // S_t at 128 * t
+  static constexpr uint32_t kTmemO = 256;                    // O_t at 256 + D * t
 };
 
 // ------------------------------------------------------------------------------------------
@@ -78,7 +89,7 @@ struct WaitCtx {
   int32_t* status;              // global, may be null
   unsigned long long limit_ns;
 };
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, int code) {
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, int code) {
   const unsigned long long t0 = global_ns();
   uint32_t spins = 0;
   while (true) {
@@ -126,21 +137,32 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
 __device__ __forceinline__ void tc_wait_ld() { __syncwarp(); asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { __syncwarp(); asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Shared-memory matrix descriptors (tcgen05), 128-byte swizzle, rows of 128 bytes, 8-row groups
+// 1024 bytes apart. Low word: start address >> 4 and (MN-major operands only) the distance between
+// 64-element spans of the MN dimension >> 4. High word: constant (8-row group stride, descriptor
+// version, swizzle mode). Stepping along a tile only ever adds a small constant to the low word.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+
 // D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
                                        uint32_t accumulate) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+      "{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %4, 0;\n"
+      "mov.b64 da, {%1, %5};\nmov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
                                        uint32_t accumulate) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+      "{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %4, 0;\n"
+      "mov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
 }
 
 // 32 consecutive fp32 columns of this thread's TMEM lane.
@@ -168,6 +190,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
         "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  __syncwarp();
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   __syncwarp();
   asm volatile(
@@ -183,86 +214,136 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);     // .x (low 16 bits) = lo
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Shared-memory matrix descriptors (tcgen05), 128-byte swizzle, rows of 128 bytes, 8-row groups
-// 1024 bytes apart. `lbo_bytes` is the distance between 64-element spans of the MN dimension
-// (only read for MN-major operands).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-         ((uint64_t)(1024u >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
 // Instruction descriptor: fp32 accumulate, bf16 A and B, A K-major, M = 128.
 __host__ __device__ constexpr uint32_t instr_desc(uint32_t n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) |
          ((128u >> 4) << 24);
 }
 
+#ifdef PP_PROFILE
+// Debug-only cycle accounting (separate build with -DPP_PROFILE; not part of the product library).
+__device__ long long g_prof[160 * 32];
+#define PROF_DECL(n) long long prof_acc[n] = {}; long long prof_t = clock64()
+#define PROF_LAP(i) do { const long long now_ = clock64(); prof_acc[i] += now_ - prof_t; prof_t = now_; } while (0)
+#define PROF_STORE(base, n) do { if (blockIdx.x < 160) for (int i_ = 0; i_ < (n); ++i_) g_prof[blockIdx.x * 32 + (base) + i_] = prof_acc[i_]; } while (0)
+#else
+#define PROF_DECL(n)
+#define PROF_LAP(i)
+#define PROF_STORE(base, n)
+#endif
+
 struct AttnArgs {
   const int32_t* table;
+  int32_t* counter;              // global work counter (a header word of the table)
   int32_t off_bin_seg_ptr, off_bin_used, off_seg_start, off_items;
+  int32_t n_items;               // geometry entries in the work list
+  int32_t subs;                  // work indices per (KV head, geometry entry)
+  int32_t pair_heads;            // 1: slots are two query heads; 0: two row tiles of one head
   int32_t group;                 // query heads per KV head
+  int32_t n_q_heads;
+  int32_t capacity;              // rows per bin
+  int32_t total_work;            // n_kv_heads * n_items * subs
   float scale_log2;              // softmax scale * log2(e)
+  __nv_bfloat16* o;
   int32_t* status;
   unsigned long long wait_limit_ns;
 };
 
-enum WaitCode { kWaitQ = 1, kWaitKFull, kWaitVFull, kWaitKEmpty, kWaitVEmpty, kWaitS, kWaitP, kWaitO };
+// What one work index means for a CTA.
+struct Work {
+  int bin, kv_row0, n, q_row0[2], jb[2], je[2], head[2], kv_head;
+  int bin_used, seg_end, key_lo[2], seg_first[2], single_seg;
+};
+
+__device__ __forceinline__ void decode_work(const AttnArgs& a, int w, Work& wk) {
+  const int sub = w % a.subs;
+  const int rest = w / a.subs;
+  const int gi = rest % a.n_items;
+  wk.kv_head = rest / a.n_items;
+  const int4* p = reinterpret_cast<const int4*>(a.table + a.off_items + kItemInts * gi);
+  const int4 x = __ldg(p), y = __ldg(p + 1);
+  wk.bin = x.x; wk.kv_row0 = x.y; wk.n = x.z; wk.q_row0[0] = x.w; wk.q_row0[1] = y.x;
+  wk.jb[0] = 0; wk.je[0] = y.z;
+  wk.jb[1] = y.y; wk.je[1] = (y.x >= 0) ? x.z : y.y;       // unused slot: empty range
+  wk.bin_used = 0;
+  if (a.pair_heads) {
+    wk.head[0] = wk.kv_head * a.group + 2 * sub;
+    wk.head[1] = wk.head[0] + 1;
+  } else {
+    wk.head[0] = wk.head[1] = wk.kv_head * a.group + sub;
+  }
+}
+
+// Second half of a work-list entry: what the softmax threads need to place their rows.
+__device__ __forceinline__ void decode_rows(const AttnArgs& a, int w, Work& wk) {
+  const int gi = (w / a.subs) % a.n_items;
+  const int4* p = reinterpret_cast<const int4*>(a.table + a.off_items + kItemInts * gi);
+  const int4 x = __ldg(p + 2), y = __ldg(p + 3);
+  wk.bin_used = x.x; wk.seg_end = x.y; wk.key_lo[0] = x.z; wk.key_lo[1] = x.w;
+  wk.seg_first[0] = y.x; wk.seg_first[1] = y.y; wk.single_seg = y.z;
+}
+
+enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWaitKFull, kWaitKEmpty,
+                kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty };
 
 template <int D>
-__global__ void __launch_bounds__(kAttnThreads, 2)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
-                 const AttnArgs args) {
+                 const __grid_constant__ CUtensorMap map_v, const AttnArgs args) {
   using Cfg = AttnCfg<D>;
-  constexpr int kStages = Cfg::kStages;
-  constexpr int kChunks = Cfg::kChunks;
+  constexpr int NK = Cfg::kKStages, NV = Cfg::kVStages, kChunks = Cfg::kChunks;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t s_q = smem_base;
-  const uint32_t s_k = s_q + Cfg::kQBytes;
-  const uint32_t s_v = s_k + kStages * Cfg::kKVBytes;
-  const uint32_t s_bar = s_v + kStages * Cfg::kKVBytes;
-  uint8_t* bar_generic = smem_raw + (s_bar - smem_u32(smem_raw));
-  // barrier slots (8 bytes each)
-  const uint32_t bar_q = s_bar + 0;
-  const uint32_t bar_s = s_bar + 8;
-  const uint32_t bar_p = s_bar + 16;
-  const uint32_t bar_o = s_bar + 24;
-  const uint32_t bar_kfull = s_bar + 32;                  // [kStages]
-  const uint32_t bar_kempty = bar_kfull + 8 * kStages;
-  const uint32_t bar_vfull = bar_kempty + 8 * kStages;
-  const uint32_t bar_vempty = bar_vfull + 8 * kStages;
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(bar_generic + 128);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(bar_generic + 132);
+  const uint32_t s_q = smem_base;                               // [2] slots
+  const uint32_t s_k = s_q + 2 * Cfg::kQBytes;                  // [NK]
+  const uint32_t s_v = s_k + NK * Cfg::kKVBytes;                // [NV]
+  const uint32_t s_misc = s_v + NV * Cfg::kKVBytes;
+  uint8_t* misc = smem_raw + (s_misc - smem_u32(smem_raw));
+  // mbarriers, 8 bytes each
+  const uint32_t bar_item_full = s_misc + 0;     // [2]
+  const uint32_t bar_item_empty = s_misc + 16;   // [2]
+  const uint32_t bar_q_full = s_misc + 32;       // [2]
+  const uint32_t bar_q_empty = s_misc + 48;      // [2]
+  const uint32_t bar_s_full = s_misc + 64;       // [2]
+  const uint32_t bar_p_full = s_misc + 80;       // [2]
+  const uint32_t bar_o_full = s_misc + 96;       // [2]
+  const uint32_t bar_o_empty = s_misc + 112;     // [2]
+  const uint32_t bar_k_full = s_misc + 128;      // [NK] (room for 8)
+  const uint32_t bar_k_empty = s_misc + 192;
+  const uint32_t bar_v_full = s_misc + 256;      // [NV] (room for 8)
+  const uint32_t bar_v_empty = s_misc + 320;
+  volatile int* s_item = reinterpret_cast<volatile int*>(misc + 384);   // [2] work index ring
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 392);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 396);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-
-  // work item
-  const int item_idx = blockIdx.x / args.group;
-  const int q_head = blockIdx.y * args.group + (blockIdx.x - item_idx * args.group);
-  const int kv_head = blockIdx.y;
-  const int4 item = *reinterpret_cast<const int4*>(args.table + args.off_items + 4 * item_idx);
-  const int bin = item.x, q_row0 = item.y, kv_row0 = item.z, n_tiles = item.w;
-
   const WaitCtx wctx{s_abort, args.status, args.wait_limit_ns};
 
   if (threadIdx.x == 0) {
-    mbar_init(bar_q, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_p, kSoftmaxThreads);
-    mbar_init(bar_o, 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar_kfull + 8 * s, 1);
-      mbar_init(bar_kempty + 8 * s, 1);
-      mbar_init(bar_vfull + 8 * s, 1);
-      mbar_init(bar_vempty + 8 * s, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_item_full + 8 * i, 1);
+      mbar_init(bar_item_empty + 8 * i, 1 + 2 * kSoftmaxThreads);
+      mbar_init(bar_q_full + 8 * i, 1);
+      mbar_init(bar_q_empty + 8 * i, 1);
+      mbar_init(bar_s_full + 8 * i, 1);
+      mbar_init(bar_p_full + 8 * i, kSoftmaxThreads);
+      mbar_init(bar_o_full + 8 * i, 1);
+      mbar_init(bar_o_empty + 8 * i, kSoftmaxThreads);
     }
+    for (int s = 0; s < NK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
+    for (int s = 0; s < NV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -275,206 +356,367 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem_base;
-  const uint32_t tmem_s = tmem_base + kTmemColS;
-  const uint32_t tmem_o = tmem_base + kTmemColO;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      mbar_expect_tx(bar_q, Cfg::kQBytes);
-      for (int c = 0; c < kChunks; ++c)
-        tma_load_4d(s_q + c * (BM * 128), &map_q, bar_q, c * 64, q_head, q_row0, bin);
-      for (int j = 0; j < n_tiles; ++j) {
-        const int s = j % kStages;
-        const uint32_t use = (uint32_t)(j / kStages);
-        const int kv0 = kv_row0 + j * BN;
-        if (!mbar_wait(bar_kempty + 8 * s, (use & 1u) ^ 1u, wctx, kWaitKEmpty)) break;
-        mbar_expect_tx(bar_kfull + 8 * s, Cfg::kKVBytes);
-        for (int c = 0; c < kChunks; ++c)
-          tma_load_4d(s_k + s * Cfg::kKVBytes + c * (BN * 128), &map_k, bar_kfull + 8 * s,
-                      c * 64, kv_head, kv0, bin);
-        if (!mbar_wait(bar_vempty + 8 * s, (use & 1u) ^ 1u, wctx, kWaitVEmpty)) break;
-        mbar_expect_tx(bar_vfull + 8 * s, Cfg::kKVBytes);
-        for (int c = 0; c < kChunks; ++c)
-          tma_load_4d(s_v + s * Cfg::kKVBytes + c * (BN * 128), &map_v, bar_vfull + 8 * s,
-                      c * 64, kv_head, kv0, bin);
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    if (warp == 0 && lane == 0) {
+      // ---------------------------------------------------------------- producer
+      uint32_t it_n = 0, kc = 0, vc = 0;
+      Work wk;
+      while (true) {
+        int w = atomicAdd(args.counter, 1);
+        if (w >= args.total_work) w = -1;
+        const uint32_t ring = it_n & 1u;
+        if (!mbar_wait(bar_item_empty + 8 * ring, ((it_n >> 1) & 1u) ^ 1u, wctx, kWaitItemEmpty)) break;
+        s_item[ring] = w;
+        mbar_arrive(bar_item_full + 8 * ring);
+        if (w < 0) break;
+        decode_work(args, w, wk);
+        bool ok = true;
+        for (int t = 0; t < 2 && ok; ++t) {
+          ok = mbar_wait(bar_q_empty + 8 * t, (it_n & 1u) ^ 1u, wctx, kWaitQEmpty);
+          if (!ok) break;
+          if (wk.jb[t] < wk.je[t]) {
+            mbar_expect_tx(bar_q_full + 8 * t, Cfg::kQBytes);
+            for (int c = 0; c < kChunks; ++c)
+              tma_load_4d(s_q + t * Cfg::kQBytes + c * (BM * 128), &map_q, bar_q_full + 8 * t,
+                          c * 64, wk.head[t], wk.q_row0[t], wk.bin);
+          } else {
+            mbar_arrive(bar_q_full + 8 * t);
+          }
+        }
+        for (int j = 0; ok && j < wk.n; ++j) {
+          const int kv0 = wk.kv_row0 + j * BN;
+          uint32_t s = kc % NK;
+          ok = mbar_wait(bar_k_empty + 8 * s, ((kc / NK) & 1u) ^ 1u, wctx, kWaitKEmpty);
+          if (!ok) break;
+          mbar_expect_tx(bar_k_full + 8 * s, Cfg::kKVBytes);
+          for (int c = 0; c < kChunks; ++c)
+            tma_load_4d(s_k + s * Cfg::kKVBytes + c * (BN * 128), &map_k, bar_k_full + 8 * s,
+                        c * 64, wk.kv_head, kv0, wk.bin);
+          ++kc;
+          s = vc % NV;
+          ok = mbar_wait(bar_v_empty + 8 * s, ((vc / NV) & 1u) ^ 1u, wctx, kWaitVEmpty);
+          if (!ok) break;
+          mbar_expect_tx(bar_v_full + 8 * s, Cfg::kKVBytes);
+          for (int c = 0; c < kChunks; ++c)
+            tma_load_4d(s_v + s * Cfg::kKVBytes + c * (BN * 128), &map_v, bar_v_full + 8 * s,
+                        c * 64, wk.kv_head, kv0, wk.bin);
+          ++vc;
+        }
+        if (!ok) break;
+        ++it_n;
       }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    } else if (warp == 1 && lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer
+      // Kept lean on purpose: one thread feeds the tensor pipe, so every scalar instruction
+      // between two tcgen05.mma counts. Descriptor low words are precomputed; inside a group of
+      // MMAs only compile-time constants are added.
       constexpr uint32_t idesc_qk = instr_desc(BN, false);
       constexpr uint32_t idesc_pv = instr_desc(D, true);
-      bool ok = mbar_wait(bar_q, 0, wctx, kWaitQ);
-      for (int j = 0; ok && j < n_tiles; ++j) {
-        const int s = j % kStages;
-        const uint32_t use = (uint32_t)(j / kStages);
-        // S = Q K^T
-        if (!mbar_wait(bar_kfull + 8 * s, use & 1u, wctx, kWaitKFull)) break;
+      const uint32_t q_lo0 = desc_lo(s_q, 0), k_lo0 = desc_lo(s_k, 0), v_lo0 = desc_lo(s_v, BN * 128);
+      uint32_t it_n = 0, kc0 = 0, vc0 = 0, tc0 = 0, tc1 = 0;
+      int n = 0, je0 = 0, jb1 = 0, je1 = 0;
+      bool ok = true;
+      PROF_DECL(8);
+      // S_t = Q_t K_j^T; the K stage is released after the last slot that reads it
+      auto issue_qk = [&](const int t, const int j) -> bool {
+        const uint32_t kc = kc0 + (uint32_t)j, s = kc % NK;
+        PROF_LAP(7);
+        if (!mbar_wait(bar_k_full + 8 * s, (kc / NK) & 1u, wctx, kWaitKFull)) return false;
+        PROF_LAP(2);
         tc_fence_after();
+        const uint32_t d = tmem_base + Cfg::kTmemS + 128u * t;
+        const uint32_t a_lo = q_lo0 + (uint32_t)t * (Cfg::kQBytes >> 4);
+        const uint32_t b_lo = k_lo0 + s * (Cfg::kKVBytes >> 4);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t koff = (uint32_t)(kk >> 2) * (BM * 128) + (uint32_t)(kk & 3) * 32;
-          mma_ss(tmem_s, smem_desc(s_q + koff, 0), smem_desc(s_k + s * Cfg::kKVBytes + koff, 0),
-                 idesc_qk, kk > 0);
+          constexpr uint32_t kChunkQ = (BM * 128) >> 4, kChunkK = (BN * 128) >> 4;
+          mma_ss(d, a_lo + (uint32_t)(kk >> 2) * kChunkQ + (uint32_t)(kk & 3) * 2,
+                 b_lo + (uint32_t)(kk >> 2) * kChunkK + (uint32_t)(kk & 3) * 2, idesc_qk, kk > 0 ? 1u : 0u);
         }
-        tc_commit(bar_kempty + 8 * s);       // K tile consumed
-        tc_commit(bar_s);                    // S ready (also: every earlier MMA has finished)
-        // O += P V
-        if (!mbar_wait(bar_p, (uint32_t)j & 1u, wctx, kWaitP)) break;
-        if (!mbar_wait(bar_vfull + 8 * s, use & 1u, wctx, kWaitVFull)) break;
-        tc_fence_after();
+        if (t == 1 || !(j >= jb1 && j < je1)) tc_commit(bar_k_empty + 8 * s);
+        tc_commit(bar_s_full + 8 * t);
+        PROF_LAP(3);
+        return true;
+      };
+      // O_t (+)= P_t V_j, then either the next S_t or the end-of-item signals of slot t
+      auto slot_step = [&](const int t, const int j, const int jb, const int je, uint32_t& tcount) -> bool {
+        if (j >= jb && j < je) {
+          const bool first = (j == jb);
+          PROF_LAP(7);
+          // the previous item's epilogue must have read O_t before it is overwritten
+          if (first && !mbar_wait(bar_o_empty + 8 * t, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty)) return false;
+          PROF_LAP(4);
+          if (!mbar_wait(bar_p_full + 8 * t, tcount & 1u, wctx, kWaitP)) return false;
+          PROF_LAP(5);
+          const uint32_t vc = vc0 + (uint32_t)j, s = vc % NV;
+          if (!mbar_wait(bar_v_full + 8 * s, (vc / NV) & 1u, wctx, kWaitVFull)) return false;
+          PROF_LAP(6);
+          tc_fence_after();
+          const uint32_t a = tmem_base + Cfg::kTmemS + 128u * t;
+          const uint32_t d = tmem_base + Cfg::kTmemO + (uint32_t)D * t;
+          const uint32_t b_lo = v_lo0 + s * (Cfg::kKVBytes >> 4);
+          mma_ts(d, a, b_lo, idesc_pv, first ? 0u : 1u);
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk) {
-          mma_ts(tmem_o, tmem_s + kk * 8,
-                 smem_desc(s_v + s * Cfg::kKVBytes + kk * (16 * 128), BN * 128), idesc_pv,
-                 (j > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 1; kk < BN / 16; ++kk)
+            mma_ts(d, a + kk * 8, b_lo + (uint32_t)kk * ((16 * 128) >> 4), idesc_pv, 1u);
+          ++tcount;
+          if (t == 1 || !(j >= jb1 && j < je1)) tc_commit(bar_v_empty + 8 * s);
+          if (j + 1 < je) return issue_qk(t, j + 1);
+          tc_commit(bar_q_empty + 8 * t);      // slot t is done with this item
+          tc_commit(bar_o_full + 8 * t);
+          return true;
         }
-        tc_commit(bar_vempty + 8 * s);       // V tile consumed
-        if (j == n_tiles - 1) tc_commit(bar_o);
+        if (j + 1 == jb && jb < je) return issue_qk(t, j + 1);   // slot t joins the key loop at the next tile
+        return true;
+      };
+      while (ok) {
+        const uint32_t ring = it_n & 1u;
+        PROF_LAP(7);
+        if (!mbar_wait(bar_item_full + 8 * ring, (it_n >> 1) & 1u, wctx, kWaitItemFull)) break;
+        const int w = s_item[ring];
+        mbar_arrive(bar_item_empty + 8 * ring);
+        if (w < 0) break;
+        {
+          Work wk;
+          decode_work(args, w, wk);
+          n = wk.n; je0 = wk.je[0]; jb1 = wk.jb[1]; je1 = wk.je[1];
+        }
+        PROF_LAP(0);
+        ok = mbar_wait(bar_q_full + 0, it_n & 1u, wctx, kWaitQFull) &&
+             mbar_wait(bar_q_full + 8, it_n & 1u, wctx, kWaitQFull);
+        if (!ok) break;
+        PROF_LAP(1);
+        if (je0 > 0) ok = issue_qk(0, 0);
+        if (ok && jb1 == 0 && je1 > 0) ok = issue_qk(1, 0);
+        for (int j = 0; ok && j < n; ++j) {
+          ok = slot_step(0, j, 0, je0, tc0);
+          if (ok) ok = slot_step(1, j, jb1, je1, tc1);
+        }
+        if (!ok) break;
+        if (je0 <= 0) {                        // unused slot: keep its per-item barriers in step
+          mbar_arrive(bar_q_empty + 0);
+          mbar_arrive(bar_o_full + 0);
+        }
+        if (jb1 >= je1) {
+          mbar_arrive(bar_q_empty + 8);
+          mbar_arrive(bar_o_full + 8);
+        }
+        kc0 += (uint32_t)n;
+        vc0 += (uint32_t)n;
+        ++it_n;
       }
+      PROF_STORE(0, 8);
     }
   } else {
-    // ------------------------------------------------------------------ softmax + epilogue
+    // ------------------------------------------------------------------ softmax + epilogue, slot t
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+    // Both slots run the same code (slot index at run time): the unrolled row loops are large and
+    // two copies of them would not stay resident in the instruction caches.
+    const int t = (warp >= 8) ? 1 : 0;
     const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
     const int row = quad * 32 + lane;                // query row inside the tile
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-    const int i_row = q_row0 + row;                  // bin-local query row
-    int key_lo = 1, key_hi = 0;                      // visible keys [key_lo, key_hi]; empty for padding
-    {
-      const int32_t* tb = args.table;
-      if (i_row < tb[args.off_bin_used + bin]) {
-        int lo = tb[args.off_bin_seg_ptr + bin], hi = tb[args.off_bin_seg_ptr + bin + 1] - 1;
-        while (lo < hi) {
-          const int mid = (lo + hi + 1) >> 1;
-          if (tb[args.off_seg_start + mid] <= i_row) lo = mid; else hi = mid - 1;
-        }
-        key_lo = tb[args.off_seg_start + lo];
-        key_hi = i_row;
-      }
-    }
+    const uint32_t tmem_s = tmem_base + Cfg::kTmemS + 128u * t + lane_base;
+    const uint32_t tmem_o = tmem_base + Cfg::kTmemO + (uint32_t)D * t + lane_base;
     const float c_scale = args.scale_log2;
-    float m_run = -INFINITY;      // running maximum, in scaled log2 units
-    float l_run = 0.f;            // running sum of exp2(s * c - m_run)
+    const int32_t* tb = args.table;
+    uint32_t it_n = 0, tcount = 0;
+    Work wk;
     bool ok = true;
-    uint32_t v[32];
-
-    for (int j = 0; j < n_tiles; ++j) {
-      const int kv0 = kv_row0 + j * BN;
-      const int c_lo = max(key_lo - kv0, 0);
-      const int c_hi = min(key_hi - kv0, BN - 1);          // visible columns [c_lo, c_hi]
-      const bool full = (c_lo == 0) && (c_hi == BN - 1);
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_s, (uint32_t)j & 1u, wctx, kWaitS));
-      if (!ok) break;                                       // warp-uniform
-      tc_fence_after();
-
-      // which 32-column chunks does any row of this warp need?
-      uint32_t need_mask = 0;
-#pragma unroll
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        const bool need = max(c_lo, ch * 32) <= min(c_hi, ch * 32 + 31);
-        if (__any_sync(0xffffffffu, need)) need_mask |= 1u << ch;
-      }
-
-      // pass 1: row maximum over the visible columns
-      float mx = -INFINITY;
-#pragma unroll
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        if (!(need_mask & (1u << ch))) continue;
-        tmem_ld32(tmem_s + lane_base + ch * 32, v);
-        tc_wait_ld();
-        if (full) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int col = ch * 32 + i;
-            if (col >= c_lo && col <= c_hi) mx = fmaxf(mx, __uint_as_float(v[i]));
+    PROF_DECL(12);
+    while (true) {
+      const uint32_t ring = it_n & 1u;
+      PROF_LAP(8);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n >> 1) & 1u, wctx, kWaitItemFull));
+      PROF_LAP(0);
+      if (!ok) break;
+      const int w = s_item[ring];
+      mbar_arrive(bar_item_empty + 8 * ring);
+      if (w < 0) break;
+      decode_work(args, w, wk);
+      decode_rows(args, w, wk);
+      const int jb_t = t ? wk.jb[1] : wk.jb[0], je_t = t ? wk.je[1] : wk.je[0];
+      const int q_row0_t = t ? wk.q_row0[1] : wk.q_row0[0], head_t = t ? wk.head[1] : wk.head[0];
+      const int key_lo_t = t ? wk.key_lo[1] : wk.key_lo[0], seg_first_t = t ? wk.seg_first[1] : wk.seg_first[0];
+      const bool used = jb_t < je_t;
+      const int i_row = q_row0_t + row;            // bin-local query row
+      int key_lo = 1, key_hi = 0;                      // visible keys [key_lo, key_hi]; empty for padding
+      bool row_valid = false;
+      if (used && i_row < wk.bin_used) {
+        key_lo = key_lo_t;
+        if (!((wk.single_seg >> t) & 1)) {             // several prompts in this tile: walk their starts
+          for (int sg = seg_first_t + 1; sg < wk.seg_end; ++sg) {
+            const int st = __ldg(tb + args.off_seg_start + sg);
+            if (st > i_row) break;
+            key_lo = st;
           }
         }
+        key_hi = i_row;
+        row_valid = true;
       }
-      // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
-      const float m_tile = mx * c_scale;
-      float m_new = m_run;
-      if (m_tile > m_run + 8.f) m_new = m_tile;
-      const bool rescale = (m_new != m_run) && (m_run != -INFINITY);
-      const float alpha = rescale ? fast_exp2(m_run - m_new) : 1.f;
-      if (j > 0 && __any_sync(0xffffffffu, rescale)) {
-#pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) {
-          tmem_ld32(tmem_o + lane_base + ch * 32, v);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-          tmem_st32(tmem_o + lane_base + ch * 32, v);
-        }
-      }
-      l_run *= alpha;
-      m_run = m_new;
+      float m_run = -INFINITY;      // running maximum, in scaled log2 units
+      float l_run = 0.f;            // running sum of exp2(s * c - m_run)
 
-      // pass 2: p = exp2(s * c - m), row sum, P (bf16) over the S columns
-      float sum = 0.f;
+      for (int j = jb_t; j < je_t; ++j) {
+        const int kv0 = wk.kv_row0 + j * BN;
+        const int c_lo = max(key_lo - kv0, 0);
+        const int c_hi = min(key_hi - kv0, BN - 1);          // visible columns [c_lo, c_hi]
+        const bool full = (c_lo == 0) && (c_hi == BN - 1);
+        const bool warp_full = __all_sync(0xffffffffu, full);
+        uint32_t need_mask = 0;                              // 32-column chunks some row of the warp sees
 #pragma unroll
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        uint32_t pk[16];
-        if (need_mask & (1u << ch)) {
-          tmem_ld32(tmem_s + lane_base + ch * 32, v);
-          tc_wait_ld();
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          const bool need = max(c_lo, ch * 32) <= min(c_hi, ch * 32 + 31);
+          if (__any_sync(0xffffffffu, need)) need_mask |= 1u << ch;
+        }
+        PROF_LAP(5);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * t, tcount & 1u, wctx, kWaitS));
+        if (!ok) break;                                      // warp-uniform
+        tc_fence_after();
+        PROF_LAP(1);
+
+        // the row's 128 scores, one TMEM round trip
+        uint32_t v[BN];
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const int col = ch * 32 + i;
-            float p0 = fast_exp2(fmaf(__uint_as_float(v[i]), c_scale, -m_run));
-            float p1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), c_scale, -m_run));
-            if (!full) {
-              if (!(col >= c_lo && col <= c_hi)) p0 = 0.f;
-              if (!(col + 1 >= c_lo && col + 1 <= c_hi)) p1 = 0.f;
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          if (need_mask & (1u << ch)) {
+            tmem_ld32(tmem_s + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[ch * 32]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[ch * 32 + i] = 0xff800000u;          // -inf
+          }
+        }
+        tc_wait_ld();
+        PROF_LAP(2);
+        if (!warp_full) {
+          // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
+          // one of the two bounds (the causal diagonal, or the first tile of a prompt)
+          const bool need_hi = __any_sync(0xffffffffu, c_hi < BN - 1);
+          const bool need_lo = __any_sync(0xffffffffu, c_lo > 0);
+#pragma unroll
+          for (int ch = 0; ch < BN / 32; ++ch) {
+            if (!(need_mask & (1u << ch))) continue;
+            if (need_hi) {
+#pragma unroll
+              for (int i = ch * 32; i < ch * 32 + 32; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
             }
-            sum += p0 + p1;
-            pk[i >> 1] = pack_bf16(p0, p1);
+            if (need_lo) {
+#pragma unroll
+              for (int i = ch * 32; i < ch * 32 + 32; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
+            }
           }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) pk[i] = 0u;
         }
-        tmem_st16(tmem_s + lane_base + ch * 16, pk);
-      }
-      l_run += sum;
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_p);
-    }
+        float mx;
+        {
+          float m0 = fmax3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+          float m1 = fmax3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+          float m2 = fmax3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
+          float m3 = fmax3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
+#pragma unroll
+          for (int i = 12; i + 7 < BN; i += 8) {
+            m0 = fmax3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+            m1 = fmax3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+            m2 = fmax3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+            m3 = fmax3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+          }
+          // 12 + 8 * 14 = 124; the last four
+          m0 = fmax3(m0, __uint_as_float(v[124]), __uint_as_float(v[125]));
+          m1 = fmax3(m1, __uint_as_float(v[126]), __uint_as_float(v[127]));
+          mx = fmaxf(fmax3(m0, m1, m2), m3);
+        }
+        PROF_LAP(3);
+        // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
+        const float m_tile = mx * c_scale;
+        float m_new = m_run;
+        if (m_tile > m_run + 8.f) m_new = m_tile;
+        const bool rescale = (m_new != m_run) && (m_run != -INFINITY);
+        const float alpha = rescale ? fast_exp2(m_run - m_new) : 1.f;
+        if (j > jb_t && __any_sync(0xffffffffu, rescale)) {
+          // S_t ready implies the previous P_t V product has finished, so O_t is stable here
+#pragma unroll 1
+          for (int ch = 0; ch < D / 16; ++ch) {          // rare path: keep it small
+            uint32_t ov[16];
+            tmem_ld16(tmem_o + ch * 16, ov);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+            tmem_st16(tmem_o + ch * 16, ov);
+          }
+        }
+        PROF_LAP(9);
+        l_run *= alpha;
+        m_run = m_new;
+        const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
 
-    // epilogue: O / l -> bf16 -> shared (128-byte swizzle, the Q buffer is free by now) -> TMA
-    ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_o, 0, wctx, kWaitO));
-    if (ok) {
-      tc_fence_after();
-      const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
+        // p = exp2(s * c - m), row sum, P (bf16) written over the S columns
+        float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-      for (int ch = 0; ch < D / 32; ++ch) {
-        tmem_ld32(tmem_o + lane_base + ch * 32, v);
-        tc_wait_ld();
-        const uint32_t box = s_q + (uint32_t)(ch >> 1) * (BM * 128) + (uint32_t)row * 128;
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t pk[16];
+          if (need_mask & (1u << ch)) {
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const uint32_t c16 = (uint32_t)((ch & 1) * 4 + q4);
-          const uint32_t addr = box + ((c16 ^ ((uint32_t)row & 7u)) << 4);
-          const uint32_t w0 = pack_bf16(__uint_as_float(v[q4 * 8 + 0]) * inv_l, __uint_as_float(v[q4 * 8 + 1]) * inv_l);
-          const uint32_t w1 = pack_bf16(__uint_as_float(v[q4 * 8 + 2]) * inv_l, __uint_as_float(v[q4 * 8 + 3]) * inv_l);
-          const uint32_t w2 = pack_bf16(__uint_as_float(v[q4 * 8 + 4]) * inv_l, __uint_as_float(v[q4 * 8 + 5]) * inv_l);
-          const uint32_t w3 = pack_bf16(__uint_as_float(v[q4 * 8 + 6]) * inv_l, __uint_as_float(v[q4 * 8 + 7]) * inv_l);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+            for (int i = 0; i < 32; i += 2) {
+              const float p0 = fast_exp2(fmaf(__uint_as_float(v[ch * 32 + i]), c_scale, neg_m));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(v[ch * 32 + i + 1]), c_scale, neg_m));
+              sum0 += p0;
+              sum1 += p1;
+              pk[i >> 1] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+          }
+          tmem_st16(tmem_s + ch * 16, pk);
         }
+        const float sum = sum0 + sum1;
+        PROF_LAP(4);
+        l_run += sum;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p_full + 8 * t);
+        ++tcount;
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (!ok) break;
+
+      // epilogue: O_t / l -> bf16 -> global (16-byte stores, rows of real tokens only)
+      PROF_LAP(5);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full + 8 * t, it_n & 1u, wctx, kWaitOFull));
+      if (!ok) break;
+      PROF_LAP(6);
+      if (used) {
+        tc_fence_after();
+        const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
+        __nv_bfloat16* orow = args.o + (((int64_t)wk.bin * args.capacity + i_row) * args.n_q_heads + head_t) * D;
+        uint32_t ov[D];
+#pragma unroll
+        for (int ch = 0; ch < D / 32; ++ch) tmem_ld32(tmem_o + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[ch * 32]));
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_o_empty + 8 * t);              // O_t may be overwritten by the next item now
+        if (row_valid) {
+#pragma unroll
+          for (int q8 = 0; q8 < D / 8; ++q8) {
+            uint4 o4;
+            o4.x = pack_bf16(__uint_as_float(ov[q8 * 8 + 0]) * inv_l, __uint_as_float(ov[q8 * 8 + 1]) * inv_l);
+            o4.y = pack_bf16(__uint_as_float(ov[q8 * 8 + 2]) * inv_l, __uint_as_float(ov[q8 * 8 + 3]) * inv_l);
+            o4.z = pack_bf16(__uint_as_float(ov[q8 * 8 + 4]) * inv_l, __uint_as_float(ov[q8 * 8 + 5]) * inv_l);
+            o4.w = pack_bf16(__uint_as_float(ov[q8 * 8 + 6]) * inv_l, __uint_as_float(ov[q8 * 8 + 7]) * inv_l);
+            *reinterpret_cast<uint4*>(orow + q8 * 8) = o4;
+          }
+        }
+      } else {
+        mbar_arrive(bar_o_empty + 8 * t);
+      }
+
+      PROF_LAP(7);
+      ++it_n;
     }
-    // all four softmax warps meet here whether or not a wait gave up
-    asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
-    if (ok && !*s_abort && warp == 2 && lane == 0) {
-      for (int c = 0; c < kChunks; ++c)
-        tma_store_4d(&map_o, s_q + c * (BM * 128), c * 64, q_head, q_row0, bin);
-      tma_store_commit_and_wait();
-    }
+#ifdef PP_PROFILE
+    prof_acc[10] = tcount;
+    if (row == 0) PROF_STORE(8 + 12 * t, 12);
+#endif
   }
 
   tc_fence_before();
@@ -525,47 +767,72 @@ unsigned long long wait_limit_ns() {
   return 2000000000ull;   // 2 s
 }
 
+int sm_count() {
+  static thread_local int cached_dev = -1, cached = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (dev != cached_dev) {
+    if (cudaDeviceGetAttribute(&cached, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    cached_dev = dev;
+  }
+  return cached;
+}
+
 template <int D>
-int launch_attention_t(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
-                       const void* q, const void* k, const void* v, void* o, int32_t* device_status,
-                       cudaStream_t stream) {
+int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
+                       const void* k, const void* v, void* o, int32_t* device_status, cudaStream_t stream) {
   using Cfg = AttnCfg<D>;
-  CUtensorMap mq, mk, mv, mo;
+  CUtensorMap mq, mk, mv;
   int st;
   if ((st = make_map(&mq, q, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
   if ((st = make_map(&mk, k, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
   if ((st = make_map(&mv, v, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
-  if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
   static bool configured = false;   // per process, per template instance
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Cfg::kSmemBytes);
     if (e != cudaSuccess) return note_cuda_error((int)e, "cudaFuncSetAttribute(smem)");
-    cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     configured = true;
   }
+  const int sms = sm_count();
+  if (sms <= 0) return note_cuda_error(-1, "multiprocessor count");
   AttnArgs a;
   a.table = d_table;
+  a.counter = d_table + kHeaderCounter;
   a.off_bin_seg_ptr = L.bin_seg_ptr;
   a.off_bin_used = L.bin_used;
   a.off_seg_start = L.seg_start;
   a.off_items = L.items;
+  a.n_items = L.n_items;
   a.group = p.n_q_heads / p.n_kv_heads;
+  a.pair_heads = (a.group % 2 == 0) ? 1 : 0;
+  a.subs = a.pair_heads ? a.group / 2 : a.group;
+  a.n_q_heads = p.n_q_heads;
+  a.capacity = p.capacity;
+  const int64_t total = (int64_t)p.n_kv_heads * L.n_items * a.subs;
+  if (total > INT32_MAX) return PP_ERR_UNSUPPORTED;
+  a.total_work = (int32_t)total;
   const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)D);
   a.scale_log2 = scale * 1.4426950408889634f;
+  a.o = static_cast<__nv_bfloat16*>(o);
   a.status = device_status;
   a.wait_limit_ns = wait_limit_ns();
-  dim3 grid((unsigned)(L.n_items * a.group), (unsigned)p.n_kv_heads, 1);
-  attention_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, mo, a);
+  const unsigned grid = (unsigned)(total < sms ? total : sms);
+  attention_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, a);
   const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "attention kernel launch");
 }
 
 }  // namespace
 
-int launch_attention(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
-                     const void* q, const void* k, const void* v, void* o, int32_t* device_status,
-                     void* stream) {
+#ifdef PP_PROFILE
+extern "C" int pp_debug_read_profile(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_prof, sizeof(long long) * (size_t)n);
+}
+#endif
+
+int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
+                     const void* k, const void* v, void* o, int32_t* device_status, void* stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p.head_dim == 128) return launch_attention_t<128>(p, d_table, L, q, k, v, o, device_status, s);
   return launch_attention_t<64>(p, d_table, L, q, k, v, o, device_status, s);

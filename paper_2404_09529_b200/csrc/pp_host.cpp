@@ -164,18 +164,24 @@ extern "C" int pp_fill_position_ids(int32_t n_bins, int32_t capacity, const int3
 // Tile work list (Section 3.2: the independent mask is block lower-triangular per prompt span,
 // so a query tile only ever needs the key rows from the start of the first prompt it touches
 // up to its own last row).
+//
+// A work item feeds the two query-tile slots of one persistent CTA, which share one stream of
+// key/value tiles. With an even number of query heads per KV head the two slots are two query
+// heads over the same 128 rows (identical key ranges); otherwise they are two consecutive
+// 128-row tiles of one head, slot 1 joining the key loop at tile jb1 and slot 0 leaving it after
+// its diagonal tile je0 - 1.
 // ------------------------------------------------------------------------------------------
 namespace pp {
 
 size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k) {
   const int64_t q_tiles = (int64_t)n_bins * ((capacity + kTileM - 1) / kTileM);
-  // header + bin_seg_ptr + bin_used + seg_start + items (4 ints each), each block 4-int aligned
+  // header + bin_seg_ptr + bin_used + seg_start + items (8 ints each), each block 4-int aligned
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
-  return (size_t)(kHeaderInts + up4(n_bins + 1) + up4(n_bins) + up4(k) + 4 * q_tiles);
+  return (size_t)(kHeaderInts + up4(n_bins + 1) + up4(n_bins) + up4(k) + kItemInts * q_tiles);
 }
 
 int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
-                         const int32_t* seg_start, const int32_t* seg_len, int32_t k,
+                         const int32_t* seg_start, const int32_t* seg_len, int32_t k, bool pair_rows,
                          int32_t* out, size_t out_ints, TableLayout* layout) {
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
   TableLayout L;
@@ -187,31 +193,68 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   std::memset(out, 0, sizeof(int32_t) * (size_t)L.items);
   std::memcpy(out + L.bin_seg_ptr, bin_seg_ptr, sizeof(int32_t) * (size_t)(n_bins + 1));
   std::memcpy(out + L.seg_start, seg_start, sizeof(int32_t) * (size_t)k);
-  struct Item { int32_t bin, q_row0, kv_row0, n_kv_tiles; };
-  std::vector<Item> items;
+  std::vector<WorkItem> items;
   try {
     for (int32_t b = 0; b < n_bins; ++b) {
       const int32_t s_lo = bin_seg_ptr[b], s_hi = bin_seg_ptr[b + 1];
       const int32_t used = seg_start[s_hi - 1] + seg_len[s_hi - 1];
       out[L.bin_used + b] = used;
       int32_t s = s_lo;
-      for (int32_t q0 = 0; q0 < used; q0 += kTileM) {
+      // first key row (rounded down to a key tile) that query tile q0 can see
+      auto kv_lo_of = [&](int32_t q0) {
         while (s + 1 < s_hi && seg_start[s + 1] <= q0) ++s;       // segment holding row q0
-        const int32_t kv_lo = (seg_start[s] / kTileN) * kTileN;
-        const int32_t kv_end = std::min(q0 + kTileM, used);
-        items.push_back({b, q0, kv_lo, (kv_end - kv_lo + kTileN - 1) / kTileN});
+        return (seg_start[s] / kTileN) * kTileN;
+      };
+      const int32_t step = pair_rows ? 2 * kTileM : kTileM;
+      for (int32_t q0 = 0; q0 < used; q0 += step) {
+        WorkItem it{};
+        it.bin = b;
+        it.kv_row0 = kv_lo_of(q0);
+        it.q_row0[0] = q0;
+        if (!pair_rows) {                       // two heads, same rows
+          it.q_row0[1] = q0;
+          it.n_kv_tiles = (std::min(q0 + kTileM, used) - it.kv_row0 + kTileN - 1) / kTileN;
+          it.jb1 = 0;
+          it.je0 = it.n_kv_tiles;
+        } else if (q0 + kTileM < used) {        // two consecutive row tiles
+          const int32_t q1 = q0 + kTileM;
+          it.q_row0[1] = q1;
+          it.jb1 = (kv_lo_of(q1) - it.kv_row0) / kTileN;
+          it.je0 = (q1 - it.kv_row0) / kTileN;  // slot 0 ends with its diagonal tile
+          it.n_kv_tiles = (std::min(q1 + kTileM, used) - it.kv_row0 + kTileN - 1) / kTileN;
+        } else {                                // last, unpaired row tile of the bin
+          it.q_row0[1] = -1;
+          it.n_kv_tiles = (used - it.kv_row0 + kTileN - 1) / kTileN;
+          it.jb1 = it.n_kv_tiles;
+          it.je0 = it.n_kv_tiles;
+        }
+        it.cost = it.je0 + (it.q_row0[1] >= 0 ? it.n_kv_tiles - it.jb1 : 0);
+        it.bin_used = used;
+        it.seg_end = s_hi;
+        for (int t = 0; t < 2; ++t) {
+          const int32_t q = it.q_row0[t];
+          if (q < 0) continue;
+          int32_t sf = s_lo;                    // segment holding row q (bins hold few segments)
+          while (sf + 1 < s_hi && seg_start[sf + 1] <= q) ++sf;
+          it.seg_first[t] = sf;
+          it.key_lo[t] = seg_start[sf];
+          const int32_t last_row = std::min(q + kTileM, used) - 1;
+          if (sf + 1 >= s_hi || seg_start[sf + 1] > last_row) it.single_seg |= 1 << t;
+        }
+        items.push_back(it);
       }
     }
-    // Longest first so that the hardware block scheduler, which hands out blocks in index
-    // order, does longest-processing-time-first scheduling; ties keep bin/row order.
+    // Longest first: CTAs draw items in list order, which gives longest-processing-time-first
+    // scheduling; ties keep bin/row order.
     std::stable_sort(items.begin(), items.end(),
-                     [](const Item& a, const Item& b) { return a.n_kv_tiles > b.n_kv_tiles; });
+                     [](const WorkItem& a, const WorkItem& b) { return a.cost > b.cost; });
   } catch (const std::bad_alloc&) {
     return PP_ERR_NO_MEMORY;
   }
-  std::memcpy(out + L.items, items.data(), sizeof(Item) * items.size());
+  static_assert(sizeof(WorkItem) == kItemInts * sizeof(int32_t), "work item layout");
+  std::memcpy(out + L.items, items.data(), sizeof(WorkItem) * items.size());
   L.n_items = (int32_t)items.size();
-  out[0] = 0x50504b31;  // "PPK1"
+  out[0] = 0x50504b32;  // "PPK2"
   out[1] = L.n_items;
   out[2] = n_bins;
   out[3] = capacity;
@@ -221,9 +264,10 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   out[7] = L.seg_start;
   out[8] = L.items;
   int64_t tiles = 0;
-  for (const Item& it : items) tiles += it.n_kv_tiles;
+  for (const WorkItem& it : items) tiles += it.cost;
   out[9] = (int32_t)std::min<int64_t>(tiles, INT32_MAX);
-  L.total_ints = (int32_t)(L.items + 4 * (int64_t)items.size());
+  out[kHeaderCounter] = 0;   // work counter the CTAs draw from; reset by every upload
+  L.total_ints = (int32_t)(L.items + kItemInts * (int64_t)items.size());
   if (layout) *layout = L;
   return PP_OK;
 }

@@ -12,6 +12,25 @@ namespace pp {
 constexpr int kTileM = 128;      // query rows per work item (tcgen05 MMA M)
 constexpr int kTileN = 128;      // key rows per inner step (tcgen05 MMA N of Q.K^T)
 constexpr int kHeaderInts = 16;  // table header, see build_prefill_tables
+constexpr int kHeaderCounter = 10;   // header word the persistent CTAs draw work indices from
+constexpr int kItemInts = 16;
+
+// One entry of the attention work list: two query-tile slots sharing one key/value tile stream.
+struct WorkItem {
+  int32_t bin;
+  int32_t kv_row0;      // first key row of the stream (multiple of kTileN)
+  int32_t n_kv_tiles;   // key tiles in the stream
+  int32_t q_row0[2];    // first query row of each slot; -1 = slot unused
+  int32_t jb1;          // slot 1 takes part in key tiles [jb1, n_kv_tiles)
+  int32_t je0;          // slot 0 takes part in key tiles [0, je0)
+  int32_t cost;         // (slot, key tile) steps, for longest-first ordering
+  int32_t bin_used;     // occupied rows of the bin
+  int32_t seg_end;      // one past the bin's last segment index
+  int32_t key_lo[2];    // start row of the prompt that holds the slot's first query row
+  int32_t seg_first[2]; // segment index of that prompt
+  int32_t single_seg;   // bit t set: all real rows of slot t belong to that one prompt
+  int32_t reserved;
+};
 
 // Offsets (in int32 units) of the blocks inside the prefill table that is built on the host and
 // copied to the device workspace.
@@ -19,7 +38,7 @@ struct TableLayout {
   int32_t bin_seg_ptr = 0;  // [R+1]
   int32_t bin_used = 0;     // [R]   occupied rows per bin
   int32_t seg_start = 0;    // [k]   bin-local first row of each segment
-  int32_t items = 0;        // [n_items][4] = (bin, q_row0, kv_row0, n_kv_tiles), longest first
+  int32_t items = 0;        // [n_items] WorkItem, longest first
   int32_t n_items = 0;
   int32_t total_ints = 0;
 };
@@ -28,7 +47,7 @@ int validate_packing(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_pt
                      const int32_t* seg_start, const int32_t* seg_len, int32_t k);
 size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k);
 int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
-                         const int32_t* seg_start, const int32_t* seg_len, int32_t k,
+                         const int32_t* seg_start, const int32_t* seg_len, int32_t k, bool pair_rows,
                          int32_t* out, size_t out_ints, TableLayout* layout);
 
 // Records a failed CUDA call for pp_last_cuda_error(); returns PP_ERR_CUDA.
@@ -37,7 +56,7 @@ int note_cuda_error(int cuda_error, const char* what);
 // Kernel launchers (device pointers, stream = cudaStream_t as void*). Return a PP_* status.
 int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
                 void* q, void* k, void* stream);
-int launch_attention(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
+int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayout& L,
                      const void* q, const void* k, const void* v, void* o,
                      int32_t* device_status, void* stream);
 int launch_unpack(const pp_attn_params& p, const int32_t* d_table, int32_t k, int64_t total_tokens,
