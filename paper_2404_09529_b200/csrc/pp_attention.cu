@@ -39,15 +39,19 @@ constexpr int kSoftmaxThreads = 128;       // per slot
 constexpr uint32_t kTmemCols = 512;
 constexpr int kRegsSoftmax = 200;          // setmaxnreg budgets: 128*104 + 256*200 <= 65536
 constexpr int kRegsOther = 104;
+constexpr uint32_t kRing = 4;               // decoded work items in flight between the fetching thread and its readers
+constexpr int kRingInts = 20;              // ints per ring entry
 
 template <int D> struct AttnCfg {
-  static constexpr int kKStages = (D == 128) ? 3 : 4;
+  static constexpr int kKStages = (D == 128) ? 2 : 4;
   static constexpr int kVStages = (D == 128) ? 2 : 4;
   static constexpr int kChunks = D / 64;                     // 128-byte swizzle spans per row
   static constexpr int kQBytes = BM * D * 2;                 // per slot
   static constexpr int kKVBytes = BN * D * 2;
-  static constexpr int kMiscBytes = 512;
-  static constexpr int kSmemBytes = 1024 /*alignment slack*/ + 2 * kQBytes + (kKStages + kVStages) * kKVBytes + kMiscBytes;
+  static constexpr int kStageOBytes = BM * 128;              // per slot: one 64-column box of O
+  static constexpr int kMiscBytes = 1024;
+  static constexpr int kSmemBytes = 1024 /*alignment slack*/ + 2 * kQBytes + (kKStages + kVStages) * kKVBytes +
+                                    2 * kStageOBytes + kMiscBytes;
   static constexpr uint32_t kTmemS = 0;                      // S_t at 128 * t
   static constexpr uint32_t kTmemO = 256;                    // O_t at 256 + D * t
 };
@@ -124,8 +128,7 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
       ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
-__device__ __forceinline__ void tma_store_commit_and_wait() {
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+__device__ __forceinline__ void tma_store_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
@@ -219,6 +222,29 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
+// Packed pairs of fp32 (sm_100 f32x2 arithmetic): halves the FMA-pipe instruction count of the
+// softmax inner loop.
+__device__ __forceinline__ uint64_t pack_f2(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack_f2(uint64_t x, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(x));
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);     // .x (low 16 bits) = lo
   return *reinterpret_cast<uint32_t*>(&h);
@@ -293,13 +319,24 @@ __device__ __forceinline__ void decode_rows(const AttnArgs& a, int w, Work& wk) 
   wk.seg_first[0] = y.x; wk.seg_first[1] = y.y; wk.single_seg = y.z;
 }
 
+// The fetching thread decodes an item once and publishes it in shared memory; every other role
+// reads it from there instead of going back to global memory.
+__device__ __forceinline__ void ring_write(volatile int* e, int w, const Work& wk) {
+  e[0] = w; e[1] = wk.bin; e[2] = wk.kv_row0; e[3] = wk.n;
+  e[4] = wk.q_row0[0]; e[5] = wk.q_row0[1]; e[6] = wk.jb[1]; e[7] = wk.je[0];
+  e[8] = wk.je[1]; e[9] = wk.head[0]; e[10] = wk.head[1]; e[11] = wk.kv_head;
+  e[12] = wk.bin_used; e[13] = wk.seg_end; e[14] = wk.key_lo[0]; e[15] = wk.key_lo[1];
+  e[16] = wk.seg_first[0]; e[17] = wk.seg_first[1]; e[18] = wk.single_seg;
+}
+
 enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWaitKFull, kWaitKEmpty,
                 kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty };
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 const __grid_constant__ CUtensorMap map_v, const AttnArgs args) {
+                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+                 const AttnArgs args) {
   using Cfg = AttnCfg<D>;
   constexpr int NK = Cfg::kKStages, NV = Cfg::kVStages, kChunks = Cfg::kChunks;
 
@@ -308,33 +345,37 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const uint32_t s_q = smem_base;                               // [2] slots
   const uint32_t s_k = s_q + 2 * Cfg::kQBytes;                  // [NK]
   const uint32_t s_v = s_k + NK * Cfg::kKVBytes;                // [NV]
-  const uint32_t s_misc = s_v + NV * Cfg::kKVBytes;
+  const uint32_t s_stage_o = s_v + NV * Cfg::kKVBytes;         // [2] slots, epilogue staging
+  const uint32_t s_misc = s_stage_o + 2 * Cfg::kStageOBytes;
   uint8_t* misc = smem_raw + (s_misc - smem_u32(smem_raw));
   // mbarriers, 8 bytes each
-  const uint32_t bar_item_full = s_misc + 0;     // [2]
-  const uint32_t bar_item_empty = s_misc + 16;   // [2]
-  const uint32_t bar_q_full = s_misc + 32;       // [2]
-  const uint32_t bar_q_empty = s_misc + 48;      // [2]
-  const uint32_t bar_s_full = s_misc + 64;       // [2]
-  const uint32_t bar_p_full = s_misc + 80;       // [2]
-  const uint32_t bar_o_full = s_misc + 96;       // [2]
-  const uint32_t bar_o_empty = s_misc + 112;     // [2]
-  const uint32_t bar_k_full = s_misc + 128;      // [NK] (room for 8)
-  const uint32_t bar_k_empty = s_misc + 192;
-  const uint32_t bar_v_full = s_misc + 256;      // [NV] (room for 8)
-  const uint32_t bar_v_empty = s_misc + 320;
-  volatile int* s_item = reinterpret_cast<volatile int*>(misc + 384);   // [2] work index ring
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 392);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 396);
+  const uint32_t bar_item_full = s_misc + 0;     // [kRing]
+  const uint32_t bar_item_empty = s_misc + 32;   // [kRing]
+  const uint32_t bar_q_full = s_misc + 64;       // [2]
+  const uint32_t bar_q_empty = s_misc + 80;      // [2]
+  const uint32_t bar_s_full = s_misc + 96;       // [2]
+  const uint32_t bar_p_full = s_misc + 112;      // [2]
+  const uint32_t bar_o_full = s_misc + 128;      // [2]
+  const uint32_t bar_o_empty = s_misc + 144;     // [2]
+  const uint32_t bar_k_full = s_misc + 160;      // [NK] (room for 8)
+  const uint32_t bar_k_empty = s_misc + 224;
+  const uint32_t bar_v_full = s_misc + 288;      // [NV] (room for 8)
+  const uint32_t bar_v_empty = s_misc + 352;
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 416);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 420);
+  volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 448);   // [kRing][kRingInts]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const WaitCtx wctx{s_abort, args.status, args.wait_limit_ns};
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < (int)kRing; ++i) {
       mbar_init(bar_item_full + 8 * i, 1);
-      mbar_init(bar_item_empty + 8 * i, 1 + 2 * kSoftmaxThreads);
+      // readers of a ring entry: the MMA thread, the two Q loaders, all softmax threads
+      mbar_init(bar_item_empty + 8 * i, 1 + 2 + 2 * kSoftmaxThreads);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(bar_q_full + 8 * i, 1);
       mbar_init(bar_q_empty + 8 * i, 1);
       mbar_init(bar_s_full + 8 * i, 1);
@@ -360,32 +401,24 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (warp == 0 && lane == 0) {
-      // ---------------------------------------------------------------- producer
-      uint32_t it_n = 0, kc = 0, vc = 0;
+      // ---------------------------------------------------------------- work fetch + K/V producer
+      uint32_t it_n = 0, kc = 0;
       Work wk;
       while (true) {
         int w = atomicAdd(args.counter, 1);
         if (w >= args.total_work) w = -1;
-        const uint32_t ring = it_n & 1u;
-        if (!mbar_wait(bar_item_empty + 8 * ring, ((it_n >> 1) & 1u) ^ 1u, wctx, kWaitItemEmpty)) break;
-        s_item[ring] = w;
+        if (w >= 0) {
+          decode_work(args, w, wk);
+          decode_rows(args, w, wk);
+        }
+        const uint32_t ring = it_n % kRing;
+        if (!mbar_wait(bar_item_empty + 8 * ring, ((it_n / kRing) & 1u) ^ 1u, wctx, kWaitItemEmpty)) break;
+        if (w >= 0) ring_write(s_ring + ring * kRingInts, w, wk);
+        else s_ring[ring * kRingInts] = -1;
         mbar_arrive(bar_item_full + 8 * ring);
         if (w < 0) break;
-        decode_work(args, w, wk);
         bool ok = true;
-        for (int t = 0; t < 2 && ok; ++t) {
-          ok = mbar_wait(bar_q_empty + 8 * t, (it_n & 1u) ^ 1u, wctx, kWaitQEmpty);
-          if (!ok) break;
-          if (wk.jb[t] < wk.je[t]) {
-            mbar_expect_tx(bar_q_full + 8 * t, Cfg::kQBytes);
-            for (int c = 0; c < kChunks; ++c)
-              tma_load_4d(s_q + t * Cfg::kQBytes + c * (BM * 128), &map_q, bar_q_full + 8 * t,
-                          c * 64, wk.head[t], wk.q_row0[t], wk.bin);
-          } else {
-            mbar_arrive(bar_q_full + 8 * t);
-          }
-        }
-        for (int j = 0; ok && j < wk.n; ++j) {
+        for (int j = 0; ok && j < wk.n; ++j, ++kc) {
           const int kv0 = wk.kv_row0 + j * BN;
           uint32_t s = kc % NK;
           ok = mbar_wait(bar_k_empty + 8 * s, ((kc / NK) & 1u) ^ 1u, wctx, kWaitKEmpty);
@@ -394,17 +427,40 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int c = 0; c < kChunks; ++c)
             tma_load_4d(s_k + s * Cfg::kKVBytes + c * (BN * 128), &map_k, bar_k_full + 8 * s,
                         c * 64, wk.kv_head, kv0, wk.bin);
-          ++kc;
-          s = vc % NV;
-          ok = mbar_wait(bar_v_empty + 8 * s, ((vc / NV) & 1u) ^ 1u, wctx, kWaitVEmpty);
+          s = kc % NV;
+          ok = mbar_wait(bar_v_empty + 8 * s, ((kc / NV) & 1u) ^ 1u, wctx, kWaitVEmpty);
           if (!ok) break;
           mbar_expect_tx(bar_v_full + 8 * s, Cfg::kKVBytes);
           for (int c = 0; c < kChunks; ++c)
             tma_load_4d(s_v + s * Cfg::kKVBytes + c * (BN * 128), &map_v, bar_v_full + 8 * s,
                         c * 64, wk.kv_head, kv0, wk.bin);
-          ++vc;
         }
         if (!ok) break;
+        ++it_n;
+      }
+    } else if (warp >= 2 && lane == 0) {
+      // ---------------------------------------------------------------- Q loader of slot t
+      const int t = warp - 2;
+      uint32_t it_n = 0;
+      while (true) {
+        const uint32_t ring = it_n % kRing;
+        if (!mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull)) break;
+        const volatile int* e = s_ring + ring * kRingInts;
+        const int w = e[0], bin = e[1];
+        const int q_row0 = e[4 + t], head = e[9 + t];
+        const bool used = t ? (e[6] < e[8]) : (e[7] > 0);
+        mbar_arrive(bar_item_empty + 8 * ring);
+        if (w < 0) break;
+        // the slot's last Q.K^T of the previous item must have finished reading the buffer
+        if (!mbar_wait(bar_q_empty + 8 * t, (it_n & 1u) ^ 1u, wctx, kWaitQEmpty)) break;
+        if (used) {
+          mbar_expect_tx(bar_q_full + 8 * t, Cfg::kQBytes);
+          for (int c = 0; c < kChunks; ++c)
+            tma_load_4d(s_q + t * Cfg::kQBytes + c * (BM * 128), &map_q, bar_q_full + 8 * t,
+                        c * 64, head, q_row0, bin);
+        } else {
+          mbar_arrive(bar_q_full + 8 * t);
+        }
         ++it_n;
       }
     } else if (warp == 1 && lane == 0) {
@@ -472,17 +528,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         return true;
       };
       while (ok) {
-        const uint32_t ring = it_n & 1u;
+        const uint32_t ring = it_n % kRing;
         PROF_LAP(7);
-        if (!mbar_wait(bar_item_full + 8 * ring, (it_n >> 1) & 1u, wctx, kWaitItemFull)) break;
-        const int w = s_item[ring];
+        if (!mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull)) break;
+        const volatile int* e = s_ring + ring * kRingInts;
+        const int w = e[0];
+        n = e[3]; jb1 = e[6]; je0 = e[7]; je1 = e[8];
         mbar_arrive(bar_item_empty + 8 * ring);
         if (w < 0) break;
-        {
-          Work wk;
-          decode_work(args, w, wk);
-          n = wk.n; je0 = wk.je[0]; jb1 = wk.jb[1]; je1 = wk.je[1];
-        }
         PROF_LAP(0);
         ok = mbar_wait(bar_q_full + 0, it_n & 1u, wctx, kWaitQFull) &&
              mbar_wait(bar_q_full + 8, it_n & 1u, wctx, kWaitQFull);
@@ -523,31 +576,31 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const float c_scale = args.scale_log2;
     const int32_t* tb = args.table;
     uint32_t it_n = 0, tcount = 0;
-    Work wk;
     bool ok = true;
     PROF_DECL(12);
     while (true) {
-      const uint32_t ring = it_n & 1u;
+      const uint32_t ring = it_n % kRing;
       PROF_LAP(8);
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n >> 1) & 1u, wctx, kWaitItemFull));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull));
       PROF_LAP(0);
       if (!ok) break;
-      const int w = s_item[ring];
+      const volatile int* e = s_ring + ring * kRingInts;
+      const int w = e[0];
+      const int item_bin = e[1], item_kv_row0 = e[2];
+      const int jb_t = t ? e[6] : 0, je_t = t ? e[8] : e[7];
+      const int q_row0_t = e[4 + t], head_t = e[9 + t];
+      const int bin_used = e[12], seg_end = e[13], key_lo_t = e[14 + t], seg_first_t = e[16 + t];
+      const int single_seg = e[18];
       mbar_arrive(bar_item_empty + 8 * ring);
       if (w < 0) break;
-      decode_work(args, w, wk);
-      decode_rows(args, w, wk);
-      const int jb_t = t ? wk.jb[1] : wk.jb[0], je_t = t ? wk.je[1] : wk.je[0];
-      const int q_row0_t = t ? wk.q_row0[1] : wk.q_row0[0], head_t = t ? wk.head[1] : wk.head[0];
-      const int key_lo_t = t ? wk.key_lo[1] : wk.key_lo[0], seg_first_t = t ? wk.seg_first[1] : wk.seg_first[0];
       const bool used = jb_t < je_t;
       const int i_row = q_row0_t + row;            // bin-local query row
       int key_lo = 1, key_hi = 0;                      // visible keys [key_lo, key_hi]; empty for padding
       bool row_valid = false;
-      if (used && i_row < wk.bin_used) {
+      if (used && i_row < bin_used) {
         key_lo = key_lo_t;
-        if (!((wk.single_seg >> t) & 1)) {             // several prompts in this tile: walk their starts
-          for (int sg = seg_first_t + 1; sg < wk.seg_end; ++sg) {
+        if (!((single_seg >> t) & 1)) {                // several prompts in this tile: walk their starts
+          for (int sg = seg_first_t + 1; sg < seg_end; ++sg) {
             const int st = __ldg(tb + args.off_seg_start + sg);
             if (st > i_row) break;
             key_lo = st;
@@ -560,7 +613,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       float l_run = 0.f;            // running sum of exp2(s * c - m_run)
 
       for (int j = jb_t; j < je_t; ++j) {
-        const int kv0 = wk.kv_row0 + j * BN;
+        const int kv0 = item_kv_row0 + j * BN;
         const int c_lo = max(key_lo - kv0, 0);
         const int c_hi = min(key_hi - kv0, BN - 1);          // visible columns [c_lo, c_hi]
         const bool full = (c_lo == 0) && (c_hi == BN - 1);
@@ -651,18 +704,23 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
 
         // p = exp2(s * c - m), row sum, P (bf16) written over the S columns
-        float sum0 = 0.f, sum1 = 0.f;
+        const uint64_t c2 = pack_f2(__float_as_uint(c_scale), __float_as_uint(c_scale));
+        const uint64_t negm2 = pack_f2(__float_as_uint(neg_m), __float_as_uint(neg_m));
+        uint64_t sum_a = 0ull, sum_b = 0ull;                 // two packed accumulators
 #pragma unroll
         for (int ch = 0; ch < BN / 32; ++ch) {
           uint32_t pk[16];
           if (need_mask & (1u << ch)) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float p0 = fast_exp2(fmaf(__uint_as_float(v[ch * 32 + i]), c_scale, neg_m));
-              const float p1 = fast_exp2(fmaf(__uint_as_float(v[ch * 32 + i + 1]), c_scale, neg_m));
-              sum0 += p0;
-              sum1 += p1;
+            for (int i = 0; i < 32; i += 4) {
+              float p0, p1, p2, p3;
+              unpack_f2(fma_f2(pack_f2(v[ch * 32 + i], v[ch * 32 + i + 1]), c2, negm2), p0, p1);
+              unpack_f2(fma_f2(pack_f2(v[ch * 32 + i + 2], v[ch * 32 + i + 3]), c2, negm2), p2, p3);
+              p0 = fast_exp2(p0); p1 = fast_exp2(p1); p2 = fast_exp2(p2); p3 = fast_exp2(p3);
+              sum_a = add_f2(sum_a, pack_f2(__float_as_uint(p0), __float_as_uint(p1)));
+              sum_b = add_f2(sum_b, pack_f2(__float_as_uint(p2), __float_as_uint(p3)));
               pk[i >> 1] = pack_bf16(p0, p1);
+              pk[(i >> 1) + 1] = pack_bf16(p2, p3);
             }
           } else {
 #pragma unroll
@@ -670,6 +728,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
           tmem_st16(tmem_s + ch * 16, pk);
         }
+        float sum0, sum1, sum2, sum3;
+        unpack_f2(sum_a, sum0, sum1);
+        unpack_f2(sum_b, sum2, sum3);
+        sum0 += sum2;
+        sum1 += sum3;
         const float sum = sum0 + sum1;
         PROF_LAP(4);
         l_run += sum;
@@ -686,24 +749,38 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (!ok) break;
       PROF_LAP(6);
       if (used) {
+        // O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store, 64 columns at a time
         tc_fence_after();
         const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
-        __nv_bfloat16* orow = args.o + (((int64_t)wk.bin * args.capacity + i_row) * args.n_q_heads + head_t) * D;
-        uint32_t ov[D];
+        const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes;
+        const uint32_t stage_row = stage + (uint32_t)row * 128;
 #pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) tmem_ld32(tmem_o + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[ch * 32]));
-        tc_wait_ld();
-        tc_fence_before();
-        mbar_arrive(bar_o_empty + 8 * t);              // O_t may be overwritten by the next item now
-        if (row_valid) {
+        for (int h = 0; h < D / 64; ++h) {
+          // the staging buffer is free once the previous store has read it
+          if (row == 0) tma_store_wait_read();
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + t), "n"(kSoftmaxThreads) : "memory");
+          uint32_t ov[64];
+          tmem_ld32(tmem_o + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&ov[0]));
+          tmem_ld32(tmem_o + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[32]));
+          tc_wait_ld();
+          if (h == D / 64 - 1) {
+            tc_fence_before();
+            mbar_arrive(bar_o_empty + 8 * t);          // O_t may be overwritten by the next item now
+          }
 #pragma unroll
-          for (int q8 = 0; q8 < D / 8; ++q8) {
-            uint4 o4;
-            o4.x = pack_bf16(__uint_as_float(ov[q8 * 8 + 0]) * inv_l, __uint_as_float(ov[q8 * 8 + 1]) * inv_l);
-            o4.y = pack_bf16(__uint_as_float(ov[q8 * 8 + 2]) * inv_l, __uint_as_float(ov[q8 * 8 + 3]) * inv_l);
-            o4.z = pack_bf16(__uint_as_float(ov[q8 * 8 + 4]) * inv_l, __uint_as_float(ov[q8 * 8 + 5]) * inv_l);
-            o4.w = pack_bf16(__uint_as_float(ov[q8 * 8 + 6]) * inv_l, __uint_as_float(ov[q8 * 8 + 7]) * inv_l);
-            *reinterpret_cast<uint4*>(orow + q8 * 8) = o4;
+          for (int c16 = 0; c16 < 8; ++c16) {
+            const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)row & 7u)) << 4);
+            const uint32_t w0 = pack_bf16(__uint_as_float(ov[c16 * 8 + 0]) * inv_l, __uint_as_float(ov[c16 * 8 + 1]) * inv_l);
+            const uint32_t w1 = pack_bf16(__uint_as_float(ov[c16 * 8 + 2]) * inv_l, __uint_as_float(ov[c16 * 8 + 3]) * inv_l);
+            const uint32_t w2 = pack_bf16(__uint_as_float(ov[c16 * 8 + 4]) * inv_l, __uint_as_float(ov[c16 * 8 + 5]) * inv_l);
+            const uint32_t w3 = pack_bf16(__uint_as_float(ov[c16 * 8 + 6]) * inv_l, __uint_as_float(ov[c16 * 8 + 7]) * inv_l);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + t), "n"(kSoftmaxThreads) : "memory");
+          if (row == 0) {
+            tma_store_4d(&map_o, stage, h * 64, head_t, q_row0_t, item_bin);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
         }
       } else {
@@ -713,6 +790,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       PROF_LAP(7);
       ++it_n;
     }
+    if (row == 0) tma_store_wait_read();             // staging must outlive the last store's read
 #ifdef PP_PROFILE
     prof_acc[10] = tcount;
     if (row == 0) PROF_STORE(8 + 12 * t, 12);
@@ -782,11 +860,12 @@ template <int D>
 int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
                        const void* k, const void* v, void* o, int32_t* device_status, cudaStream_t stream) {
   using Cfg = AttnCfg<D>;
-  CUtensorMap mq, mk, mv;
+  CUtensorMap mq, mk, mv, mo;
   int st;
   if ((st = make_map(&mq, q, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
   if ((st = make_map(&mk, k, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
   if ((st = make_map(&mv, v, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
+  if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
   static bool configured = false;   // per process, per template instance
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -818,7 +897,7 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   a.status = device_status;
   a.wait_limit_ns = wait_limit_ns();
   const unsigned grid = (unsigned)(total < sms ? total : sms);
-  attention_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, a);
+  attention_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, mo, a);
   const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "attention kernel launch");
 }
