@@ -4,19 +4,20 @@
 // row carries the key range [start row of its prompt, its own row], and the host work list
 // restricts each query tile to the key tiles that can intersect such a range.
 //
-// Persistent kernel, one CTA per SM, 384 threads. Each CTA draws work items from a global counter
+// Persistent kernel, one CTA per SM, 640 threads. Each CTA draws work items from a global counter
 // (items are listed KV-head-major, longest first). A work item has two 128-row query-tile slots
 // that share one stream of 128-row key/value tiles: two query heads of one KV head over the same
 // rows (even GQA group), or two consecutive row tiles of one head.
-//   warp 0       producer: draws items, TMA-loads Q (per slot) and the K / V tile rings
+//   warp 0       draws and decodes items, TMA-loads the K / V tile rings
 //   warp 1       issues tcgen05.mma: S_t = Q_t K^T into TMEM, O_t += P_t V with P_t read from TMEM;
-//                the two slots alternate (S0, S1, then PV0, S0', PV1, S1', ...) so that one slot's
-//                MMAs run while the other slot's softmax works
-//   warps 4-7    softmax of slot 0, one query row per thread (TMEM lane = row)
-//   warps 8-11   softmax of slot 1
-// Softmax: tcgen05.ld the 128 scores of the row, mask to the row's key range, lazy running maximum
-// (O is rescaled only when the maximum grows by more than 2^8), exp2, P written as bf16 over the S
-// columns, and at the end of an item O / l is stored straight to global memory.
+//                the two slots alternate so that one slot's MMAs run while the other's softmax works
+//   warps 2-3    TMA-load Q of slot 0 / slot 1
+//   warps 4-11   softmax of slot 0: two threads per query row (TMEM lane = row), one per 64-key half
+//   warps 12-19  softmax of slot 1
+// Softmax: tcgen05.ld the thread's 64 scores, mask to the row's key range, row maximum exchanged
+// between the two halves through shared memory, lazy running maximum (O is rescaled only when
+// the maximum grows by more than 2^8), exp2, P written as bf16 over the S columns; at the end of
+// an item O / l goes through a swizzled staging buffer and a TMA store.
 // TMEM: S0 | S1 | O0 | O1 = 512 columns. Every mbarrier wait is bounded.
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -34,11 +35,11 @@ namespace {
 
 constexpr int BM = kTileM;
 constexpr int BN = kTileN;
-constexpr int kAttnThreads = 384;
-constexpr int kSoftmaxThreads = 128;       // per slot
+constexpr int kAttnThreads = 640;
+constexpr int kSoftmaxThreads = 256;       // per slot: two threads per query row
 constexpr uint32_t kTmemCols = 512;
-constexpr int kRegsSoftmax = 200;          // setmaxnreg budgets: 128*104 + 256*200 <= 65536
-constexpr int kRegsOther = 104;
+constexpr int kRegsSoftmax = 104;          // setmaxnreg budgets: 640 threads start with 96 registers each;
+constexpr int kRegsOther = 64;              // warps 0-3 give back 32 each, the 512 softmax threads take 8 each
 constexpr uint32_t kRing = 4;               // decoded work items in flight between the fetching thread and its readers
 constexpr int kRingInts = 20;              // ints per ring entry
 
@@ -49,9 +50,11 @@ template <int D> struct AttnCfg {
   static constexpr int kQBytes = BM * D * 2;                 // per slot
   static constexpr int kKVBytes = BN * D * 2;
   static constexpr int kStageOBytes = BM * 128;              // per slot: one 64-column box of O
-  static constexpr int kMiscBytes = 1024;
-  static constexpr int kSmemBytes = 1024 /*alignment slack*/ + 2 * kQBytes + (kKStages + kVStages) * kKVBytes +
-                                    2 * kStageOBytes + kMiscBytes;
+  // barriers + work ring (768) and the row-maximum exchange buffer [slot][half][row] (2048), placed
+  // in front of the 1024-byte-aligned tiles; at D = 128 the total is exactly the 227 KB limit
+  static constexpr int kMiscBytes = 3072;
+  static constexpr int kTileBytes = 2 * kQBytes + (kKStages + kVStages) * kKVBytes + 2 * kStageOBytes;
+  static constexpr int kSmemBytes = kMiscBytes + kTileBytes;
   static constexpr uint32_t kTmemS = 0;                      // S_t at 128 * t
   static constexpr uint32_t kTmemO = 256;                    // O_t at 256 + D * t
 };
@@ -340,14 +343,21 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   using Cfg = AttnCfg<D>;
   constexpr int NK = Cfg::kKStages, NV = Cfg::kVStages, kChunks = Cfg::kChunks;
 
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t s_q = smem_base;                               // [2] slots
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t s_misc = smem_u32(smem_raw);
+  uint8_t* misc = smem_raw;
+  const uint32_t s_q = (s_misc + 2816u + 1023u) & ~1023u;       // [2] slots; tiles need 1024-byte alignment
   const uint32_t s_k = s_q + 2 * Cfg::kQBytes;                  // [NK]
   const uint32_t s_v = s_k + NK * Cfg::kKVBytes;                // [NV]
-  const uint32_t s_stage_o = s_v + NV * Cfg::kKVBytes;         // [2] slots, epilogue staging
-  const uint32_t s_misc = s_stage_o + 2 * Cfg::kStageOBytes;
-  uint8_t* misc = smem_raw + (s_misc - smem_u32(smem_raw));
+  const uint32_t s_stage_o = s_v + NV * Cfg::kKVBytes;          // [2] slots, epilogue staging
+  {
+    uint32_t dyn_bytes;
+    asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
+    if (s_stage_o + 2 * Cfg::kStageOBytes > s_misc + dyn_bytes) {   // base less aligned than expected
+      if (threadIdx.x == 0 && args.status) atomicCAS(args.status, 0, 100);
+      return;
+    }
+  }
   // mbarriers, 8 bytes each
   const uint32_t bar_item_full = s_misc + 0;     // [kRing]
   const uint32_t bar_item_empty = s_misc + 32;   // [kRing]
@@ -364,6 +374,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 416);
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 420);
   volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 448);   // [kRing][kRingInts]
+  volatile float* s_xchg = reinterpret_cast<volatile float*>(misc + 768);   // [2 slots][2 halves][128 rows]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -381,7 +392,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_init(bar_s_full + 8 * i, 1);
       mbar_init(bar_p_full + 8 * i, kSoftmaxThreads);
       mbar_init(bar_o_full + 8 * i, 1);
-      mbar_init(bar_o_empty + 8 * i, kSoftmaxThreads);
+      mbar_init(bar_o_empty + 8 * i, kSoftmaxThreads / 2);   // the half-0 threads run the epilogue
     }
     for (int s = 0; s < NK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
     for (int s = 0; s < NV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
@@ -563,16 +574,21 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       PROF_STORE(0, 8);
     }
   } else {
-    // ------------------------------------------------------------------ softmax + epilogue, slot t
+    // ------------------------------------------------------------------ softmax + epilogue
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-    // Both slots run the same code (slot index at run time): the unrolled row loops are large and
-    // two copies of them would not stay resident in the instruction caches.
-    const int t = (warp >= 8) ? 1 : 0;
+    // All softmax warps run the same code (slot and half at run time): the unrolled row loops are
+    // large and several copies of them would not stay resident in the instruction caches.
+    const int t = (warp - 4) >> 3;                   // slot
+    const int h = ((warp - 4) >> 2) & 1;             // which 64 keys of a 128-key tile this thread owns
     const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
     const int row = quad * 32 + lane;                // query row inside the tile
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const uint32_t tmem_s = tmem_base + Cfg::kTmemS + 128u * t + lane_base;
     const uint32_t tmem_o = tmem_base + Cfg::kTmemO + (uint32_t)D * t + lane_base;
+    volatile float* x_mine = s_xchg + (t * 2 + h) * 128 + row;
+    volatile float* x_other = s_xchg + (t * 2 + (h ^ 1)) * 128 + row;
+    const int bar_slot = 1 + t;                      // named barrier of the slot's 256 threads
+    const int bar_epi = 3 + t;                       // named barrier of the slot's 128 half-0 threads
     const float c_scale = args.scale_log2;
     const int32_t* tb = args.table;
     uint32_t it_n = 0, tcount = 0;
@@ -594,9 +610,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_arrive(bar_item_empty + 8 * ring);
       if (w < 0) break;
       const bool used = jb_t < je_t;
-      const int i_row = q_row0_t + row;            // bin-local query row
+      const int i_row = q_row0_t + row;                // bin-local query row
       int key_lo = 1, key_hi = 0;                      // visible keys [key_lo, key_hi]; empty for padding
-      bool row_valid = false;
       if (used && i_row < bin_used) {
         key_lo = key_lo_t;
         if (!((single_seg >> t) & 1)) {                // several prompts in this tile: walk their starts
@@ -607,58 +622,50 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         key_hi = i_row;
-        row_valid = true;
       }
-      float m_run = -INFINITY;      // running maximum, in scaled log2 units
-      float l_run = 0.f;            // running sum of exp2(s * c - m_run)
+      float m_run = -INFINITY;      // running maximum of the whole row, in scaled log2 units
+      float l_run = 0.f;            // this thread's share of the running sum of exp2(s * c - m_run)
 
       for (int j = jb_t; j < je_t; ++j) {
-        const int kv0 = item_kv_row0 + j * BN;
+        const int kv0 = item_kv_row0 + j * BN + 64 * h;      // first key of this thread's half
         const int c_lo = max(key_lo - kv0, 0);
-        const int c_hi = min(key_hi - kv0, BN - 1);          // visible columns [c_lo, c_hi]
-        const bool full = (c_lo == 0) && (c_hi == BN - 1);
+        const int c_hi = min(key_hi - kv0, 63);              // visible columns [c_lo, c_hi] of the half
+        const bool full = (c_lo == 0) && (c_hi == 63);
         const bool warp_full = __all_sync(0xffffffffu, full);
-        uint32_t need_mask = 0;                              // 32-column chunks some row of the warp sees
-#pragma unroll
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          const bool need = max(c_lo, ch * 32) <= min(c_hi, ch * 32 + 31);
-          if (__any_sync(0xffffffffu, need)) need_mask |= 1u << ch;
-        }
+        const bool need0 = __any_sync(0xffffffffu, c_lo <= min(c_hi, 31));
+        const bool need1 = __any_sync(0xffffffffu, max(c_lo, 32) <= c_hi);
         PROF_LAP(5);
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * t, tcount & 1u, wctx, kWaitS));
         if (!ok) break;                                      // warp-uniform
         tc_fence_after();
         PROF_LAP(1);
 
-        // the row's 128 scores, one TMEM round trip
-        uint32_t v[BN];
+        // this thread's 64 scores, one TMEM round trip
+        uint32_t v[64];
+        if (need0) {
+          tmem_ld32(tmem_s + 64 * h, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+        } else {
 #pragma unroll
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          if (need_mask & (1u << ch)) {
-            tmem_ld32(tmem_s + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[ch * 32]));
-          } else {
+          for (int i = 0; i < 32; ++i) v[i] = 0xff800000u;                    // -inf
+        }
+        if (need1) {
+          tmem_ld32(tmem_s + 64 * h + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+        } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[ch * 32 + i] = 0xff800000u;          // -inf
-          }
+          for (int i = 32; i < 64; ++i) v[i] = 0xff800000u;
         }
         tc_wait_ld();
         PROF_LAP(2);
         if (!warp_full) {
           // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
           // one of the two bounds (the causal diagonal, or the first tile of a prompt)
-          const bool need_hi = __any_sync(0xffffffffu, c_hi < BN - 1);
-          const bool need_lo = __any_sync(0xffffffffu, c_lo > 0);
+          if (__any_sync(0xffffffffu, c_hi < 63)) {
 #pragma unroll
-          for (int ch = 0; ch < BN / 32; ++ch) {
-            if (!(need_mask & (1u << ch))) continue;
-            if (need_hi) {
+            for (int i = 0; i < 64; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
+          }
+          if (__any_sync(0xffffffffu, c_lo > 0)) {
 #pragma unroll
-              for (int i = ch * 32; i < ch * 32 + 32; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
-            }
-            if (need_lo) {
-#pragma unroll
-              for (int i = ch * 32; i < ch * 32 + 32; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
-            }
+            for (int i = 0; i < 64; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
           }
         }
         float mx;
@@ -668,17 +675,22 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           float m2 = fmax3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
           float m3 = fmax3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
 #pragma unroll
-          for (int i = 12; i + 7 < BN; i += 8) {
+          for (int i = 12; i + 7 < 64; i += 8) {
             m0 = fmax3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
             m1 = fmax3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
             m2 = fmax3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
             m3 = fmax3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
           }
-          // 12 + 8 * 14 = 124; the last four
-          m0 = fmax3(m0, __uint_as_float(v[124]), __uint_as_float(v[125]));
-          m1 = fmax3(m1, __uint_as_float(v[126]), __uint_as_float(v[127]));
+          // 12 + 8 * 6 = 60; the last four
+          m0 = fmax3(m0, __uint_as_float(v[60]), __uint_as_float(v[61]));
+          m1 = fmax3(m1, __uint_as_float(v[62]), __uint_as_float(v[63]));
           mx = fmaxf(fmax3(m0, m1, m2), m3);
         }
+        // Row maximum over both halves. The barrier also orders the two halves' S reads before
+        // either writes P over the S columns.
+        *x_mine = mx;
+        asm volatile("bar.sync %0, %1;" ::"r"(bar_slot), "n"(kSoftmaxThreads) : "memory");
+        mx = fmaxf(mx, *x_other);
         PROF_LAP(3);
         // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
         const float m_tile = mx * c_scale;
@@ -687,15 +699,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const bool rescale = (m_new != m_run) && (m_run != -INFINITY);
         const float alpha = rescale ? fast_exp2(m_run - m_new) : 1.f;
         if (j > jb_t && __any_sync(0xffffffffu, rescale)) {
-          // S_t ready implies the previous P_t V product has finished, so O_t is stable here
+          // S_t ready implies the previous P_t V product has finished, so O_t is stable here;
+          // each half rescales its own D/2 columns of the row
 #pragma unroll 1
-          for (int ch = 0; ch < D / 16; ++ch) {          // rare path: keep it small
+          for (int ch = 0; ch < D / 32; ++ch) {          // rare path: keep it small
             uint32_t ov[16];
-            tmem_ld16(tmem_o + ch * 16, ov);
+            tmem_ld16(tmem_o + (D / 2) * h + ch * 16, ov);
             tc_wait_ld();
 #pragma unroll
             for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-            tmem_st16(tmem_o + ch * 16, ov);
+            tmem_st16(tmem_o + (D / 2) * h + ch * 16, ov);
           }
         }
         PROF_LAP(9);
@@ -708,9 +721,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint64_t negm2 = pack_f2(__float_as_uint(neg_m), __float_as_uint(neg_m));
         uint64_t sum_a = 0ull, sum_b = 0ull;                 // two packed accumulators
 #pragma unroll
-        for (int ch = 0; ch < BN / 32; ++ch) {
+        for (int ch = 0; ch < 2; ++ch) {
           uint32_t pk[16];
-          if (need_mask & (1u << ch)) {
+          if (ch == 0 ? need0 : need1) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
               float p0, p1, p2, p3;
@@ -726,16 +739,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
             for (int i = 0; i < 16; ++i) pk[i] = 0u;
           }
-          tmem_st16(tmem_s + ch * 16, pk);
+          tmem_st16(tmem_s + 32 * h + ch * 16, pk);
         }
         float sum0, sum1, sum2, sum3;
         unpack_f2(sum_a, sum0, sum1);
         unpack_f2(sum_b, sum2, sum3);
-        sum0 += sum2;
-        sum1 += sum3;
-        const float sum = sum0 + sum1;
         PROF_LAP(4);
-        l_run += sum;
+        l_run += (sum0 + sum2) + (sum1 + sum3);
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p_full + 8 * t);
@@ -743,57 +753,63 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       if (!ok) break;
 
-      // epilogue: O_t / l -> bf16 -> global (16-byte stores, rows of real tokens only)
+      // epilogue: O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store
       PROF_LAP(5);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full + 8 * t, it_n & 1u, wctx, kWaitOFull));
       if (!ok) break;
       PROF_LAP(6);
       if (used) {
-        // O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store, 64 columns at a time
-        tc_fence_after();
-        const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
-        const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes;
-        const uint32_t stage_row = stage + (uint32_t)row * 128;
+        // the half-1 threads hand their share of the row sum to the half-0 threads, which run the
+        // epilogue; the second barrier keeps the exchange slot from being reused too early
+        if (h == 1) *x_mine = l_run;
+        asm volatile("bar.sync %0, %1;" ::"r"(bar_slot), "n"(kSoftmaxThreads) : "memory");
+        const float l_row = (h == 0) ? l_run + *x_other : 0.f;
+        asm volatile("bar.sync %0, %1;" ::"r"(bar_slot), "n"(kSoftmaxThreads) : "memory");
+        if (h == 0) {
+          tc_fence_after();
+          const float inv_l = l_row > 0.f ? 1.f / l_row : 0.f;
+          const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes;
+          const uint32_t stage_row = stage + (uint32_t)row * 128;
+#pragma unroll 1
+          for (int hh = 0; hh < D / 64; ++hh) {          // 64 columns (one TMA box) at a time
+            // the staging buffer is free once the previous store has read it
+            if (row == 0) tma_store_wait_read();
+            asm volatile("bar.sync %0, %1;" ::"r"(bar_epi), "n"(kSoftmaxThreads / 2) : "memory");
+            uint32_t ov[64];
+            tmem_ld32(tmem_o + hh * 64, *reinterpret_cast<uint32_t(*)[32]>(&ov[0]));
+            tmem_ld32(tmem_o + hh * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[32]));
+            tc_wait_ld();
+            if (hh == D / 64 - 1) {
+              tc_fence_before();
+              mbar_arrive(bar_o_empty + 8 * t);        // O_t may be overwritten by the next item now
+            }
 #pragma unroll
-        for (int h = 0; h < D / 64; ++h) {
-          // the staging buffer is free once the previous store has read it
-          if (row == 0) tma_store_wait_read();
-          asm volatile("bar.sync %0, %1;" ::"r"(1 + t), "n"(kSoftmaxThreads) : "memory");
-          uint32_t ov[64];
-          tmem_ld32(tmem_o + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&ov[0]));
-          tmem_ld32(tmem_o + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[32]));
-          tc_wait_ld();
-          if (h == D / 64 - 1) {
-            tc_fence_before();
-            mbar_arrive(bar_o_empty + 8 * t);          // O_t may be overwritten by the next item now
-          }
-#pragma unroll
-          for (int c16 = 0; c16 < 8; ++c16) {
-            const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)row & 7u)) << 4);
-            const uint32_t w0 = pack_bf16(__uint_as_float(ov[c16 * 8 + 0]) * inv_l, __uint_as_float(ov[c16 * 8 + 1]) * inv_l);
-            const uint32_t w1 = pack_bf16(__uint_as_float(ov[c16 * 8 + 2]) * inv_l, __uint_as_float(ov[c16 * 8 + 3]) * inv_l);
-            const uint32_t w2 = pack_bf16(__uint_as_float(ov[c16 * 8 + 4]) * inv_l, __uint_as_float(ov[c16 * 8 + 5]) * inv_l);
-            const uint32_t w3 = pack_bf16(__uint_as_float(ov[c16 * 8 + 6]) * inv_l, __uint_as_float(ov[c16 * 8 + 7]) * inv_l);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
-          }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          asm volatile("bar.sync %0, %1;" ::"r"(1 + t), "n"(kSoftmaxThreads) : "memory");
-          if (row == 0) {
-            tma_store_4d(&map_o, stage, h * 64, head_t, q_row0_t, item_bin);
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            for (int c16 = 0; c16 < 8; ++c16) {
+              const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)row & 7u)) << 4);
+              const uint32_t w0 = pack_bf16(__uint_as_float(ov[c16 * 8 + 0]) * inv_l, __uint_as_float(ov[c16 * 8 + 1]) * inv_l);
+              const uint32_t w1 = pack_bf16(__uint_as_float(ov[c16 * 8 + 2]) * inv_l, __uint_as_float(ov[c16 * 8 + 3]) * inv_l);
+              const uint32_t w2 = pack_bf16(__uint_as_float(ov[c16 * 8 + 4]) * inv_l, __uint_as_float(ov[c16 * 8 + 5]) * inv_l);
+              const uint32_t w3 = pack_bf16(__uint_as_float(ov[c16 * 8 + 6]) * inv_l, __uint_as_float(ov[c16 * 8 + 7]) * inv_l);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("bar.sync %0, %1;" ::"r"(bar_epi), "n"(kSoftmaxThreads / 2) : "memory");
+            if (row == 0) {
+              tma_store_4d(&map_o, stage, hh * 64, head_t, q_row0_t, item_bin);
+              asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
           }
         }
-      } else {
+      } else if (h == 0) {
         mbar_arrive(bar_o_empty + 8 * t);
       }
-
       PROF_LAP(7);
       ++it_n;
     }
-    if (row == 0) tma_store_wait_read();             // staging must outlive the last store's read
+    if (h == 0 && row == 0) tma_store_wait_read();     // staging must outlive the last store's read
 #ifdef PP_PROFILE
     prof_acc[10] = tcount;
-    if (row == 0) PROF_STORE(8 + 12 * t, 12);
+    if (row == 0 && h == 0) PROF_STORE(8 + 12 * t, 12);
 #endif
   }
 
