@@ -81,9 +81,8 @@ extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t*
   if ((st = pp::check_device()) != PP_OK) return st;
 
   pp::TableLayout L;
-  // an even number of query heads per KV head pairs two heads per work item, else two row tiles
-  const bool pair_rows = ((params->n_q_heads / params->n_kv_heads) % 2) != 0;
-  st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k, pair_rows,
+  st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
+                                params->n_q_heads / params->n_kv_heads,
                                 static_cast<int32_t*>(host_workspace), workspace_bytes / sizeof(int32_t), &L);
   if (st != PP_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

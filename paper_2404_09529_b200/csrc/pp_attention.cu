@@ -335,7 +335,11 @@ __device__ __forceinline__ void ring_write(volatile int* e, int w, const Work& w
 enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWaitKFull, kWaitKEmpty,
                 kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty };
 
-template <int D>
+// kIndep = false: the two slots of a CTA work on one item and share its K/V stream (long
+//   sequences, GQA head pairs). kIndep = true: every slot draws its own single-tile items and loads
+//   its own K/V tiles, so neither slot ever waits for the other (short prompts, where pairing two
+//   row tiles of different length would leave one slot idle for a tile per item).
+template <int D, bool kIndep>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
@@ -346,7 +350,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t s_misc = smem_u32(smem_raw);
   uint8_t* misc = smem_raw;
-  const uint32_t s_q = (s_misc + 2816u + 1023u) & ~1023u;       // [2] slots; tiles need 1024-byte alignment
+  const uint32_t s_q = (s_misc + 3072u + 1023u) & ~1023u;       // [2] slots; tiles need 1024-byte alignment
   const uint32_t s_k = s_q + 2 * Cfg::kQBytes;                  // [NK]
   const uint32_t s_v = s_k + NK * Cfg::kKVBytes;                // [NV]
   const uint32_t s_stage_o = s_v + NV * Cfg::kKVBytes;          // [2] slots, epilogue staging
@@ -359,32 +363,35 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   }
   // mbarriers, 8 bytes each
-  const uint32_t bar_item_full = s_misc + 0;     // [kRing]
-  const uint32_t bar_item_empty = s_misc + 32;   // [kRing]
-  const uint32_t bar_q_full = s_misc + 64;       // [2]
-  const uint32_t bar_q_empty = s_misc + 80;      // [2]
-  const uint32_t bar_s_full = s_misc + 96;       // [2]
-  const uint32_t bar_p_full = s_misc + 112;      // [2]
-  const uint32_t bar_o_full = s_misc + 128;      // [2]
-  const uint32_t bar_o_empty = s_misc + 144;     // [2]
-  const uint32_t bar_k_full = s_misc + 160;      // [NK] (room for 8)
-  const uint32_t bar_k_empty = s_misc + 224;
-  const uint32_t bar_v_full = s_misc + 288;      // [NV] (room for 8)
-  const uint32_t bar_v_empty = s_misc + 352;
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 416);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 420);
-  volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 448);   // [kRing][kRingInts]
-  volatile float* s_xchg = reinterpret_cast<volatile float*>(misc + 768);   // [2 slots][2 halves][128 rows]
+  const uint32_t bar_item_full = s_misc + 0;     // [2 rings][kRing]
+  const uint32_t bar_item_empty = s_misc + 64;   // [2 rings][kRing]
+  const uint32_t bar_q_full = s_misc + 128;      // [2]
+  const uint32_t bar_q_empty = s_misc + 144;     // [2]
+  const uint32_t bar_s_full = s_misc + 160;      // [2]
+  const uint32_t bar_p_full = s_misc + 176;      // [2]
+  const uint32_t bar_o_full = s_misc + 192;      // [2]
+  const uint32_t bar_o_empty = s_misc + 208;     // [2]
+  const uint32_t bar_k_full = s_misc + 224;      // [4]
+  const uint32_t bar_k_empty = s_misc + 256;     // [4]
+  const uint32_t bar_v_full = s_misc + 288;      // [4]
+  const uint32_t bar_v_empty = s_misc + 320;     // [4]
+  volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 352);   // [2 rings][kRing][kRingInts]
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 992);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 996);
+  volatile float* s_xchg = reinterpret_cast<volatile float*>(misc + 1024);   // [2 slots][2 halves][128 rows]
+  static_assert(352 + 2 * kRing * kRingInts * 4 <= 992, "ring does not fit");
+  static_assert(NK <= 4 && NV <= 4, "barrier slots");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const WaitCtx wctx{s_abort, args.status, args.wait_limit_ns};
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < (int)kRing; ++i) {
+    for (int i = 0; i < 2 * (int)kRing; ++i) {
       mbar_init(bar_item_full + 8 * i, 1);
-      // readers of a ring entry: the MMA thread, the two Q loaders, all softmax threads
-      mbar_init(bar_item_empty + 8 * i, 1 + 2 + 2 * kSoftmaxThreads);
+      // readers of a ring entry: the MMA thread and the softmax threads of the slot(s) it feeds;
+      // in shared mode also the two Q loaders
+      mbar_init(bar_item_empty + 8 * i, kIndep ? 1 + kSoftmaxThreads : 1 + 2 + 2 * kSoftmaxThreads);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_q_full + 8 * i, 1);
@@ -411,6 +418,140 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    if constexpr (kIndep) {
+      if (warp >= 2 && lane == 0) {
+        // -------------------------------------------------------------- producer of slot t:
+        // draws the slot's own items, loads Q and the item's K / V tiles (one stage each)
+        const int t = warp - 2;
+        const uint32_t ring_bar = 8 * (uint32_t)t * kRing;
+        volatile int* ring_base = s_ring + t * (int)kRing * kRingInts;
+        uint32_t it_n = 0, kc = 0;
+        Work wk;
+        while (true) {
+          int w = atomicAdd(args.counter, 1);
+          if (w >= args.total_work) w = -1;
+          if (w >= 0) {
+            decode_work(args, w, wk);
+            decode_rows(args, w, wk);
+          }
+          const uint32_t ring = it_n % kRing;
+          if (!mbar_wait(bar_item_empty + ring_bar + 8 * ring, ((it_n / kRing) & 1u) ^ 1u, wctx, kWaitItemEmpty)) break;
+          if (w >= 0) ring_write(ring_base + ring * kRingInts, w, wk);
+          else ring_base[ring * kRingInts] = -1;
+          mbar_arrive(bar_item_full + ring_bar + 8 * ring);
+          if (w < 0) break;
+          // the slot's last Q.K^T of the previous item must have finished reading the Q buffer
+          if (!mbar_wait(bar_q_empty + 8 * t, (it_n & 1u) ^ 1u, wctx, kWaitQEmpty)) break;
+          mbar_expect_tx(bar_q_full + 8 * t, Cfg::kQBytes);
+          for (int c = 0; c < kChunks; ++c)
+            tma_load_4d(s_q + t * Cfg::kQBytes + c * (BM * 128), &map_q, bar_q_full + 8 * t,
+                        c * 64, wk.head[0], wk.q_row0[0], wk.bin);
+          bool ok = true;
+          for (int j = 0; ok && j < wk.n; ++j, ++kc) {
+            const int kv0 = wk.kv_row0 + j * BN;
+            ok = mbar_wait(bar_k_empty + 8 * t, (kc & 1u) ^ 1u, wctx, kWaitKEmpty);
+            if (!ok) break;
+            mbar_expect_tx(bar_k_full + 8 * t, Cfg::kKVBytes);
+            for (int c = 0; c < kChunks; ++c)
+              tma_load_4d(s_k + t * Cfg::kKVBytes + c * (BN * 128), &map_k, bar_k_full + 8 * t,
+                          c * 64, wk.kv_head, kv0, wk.bin);
+            ok = mbar_wait(bar_v_empty + 8 * t, (kc & 1u) ^ 1u, wctx, kWaitVEmpty);
+            if (!ok) break;
+            mbar_expect_tx(bar_v_full + 8 * t, Cfg::kKVBytes);
+            for (int c = 0; c < kChunks; ++c)
+              tma_load_4d(s_v + t * Cfg::kKVBytes + c * (BN * 128), &map_v, bar_v_full + 8 * t,
+                          c * 64, wk.kv_head, kv0, wk.bin);
+          }
+          if (!ok) break;
+          ++it_n;
+        }
+      } else if (warp == 1 && lane == 0) {
+        // -------------------------------------------------------------- MMA issuer, independent slots
+        // Each slot walks  item -> S(0) -> [P V(j), S(j+1)] ... -> end of item  on its own; the
+        // thread polls both and issues whichever next step is ready.
+        constexpr uint32_t idesc_qk = instr_desc(BN, false);
+        constexpr uint32_t idesc_pv = instr_desc(D, true);
+        const uint32_t q_lo0 = desc_lo(s_q, 0), k_lo0 = desc_lo(s_k, 0), v_lo0 = desc_lo(s_v, BN * 128);
+        enum { kNeedItem = 0, kNeedS, kNeedPV, kDone };
+        uint32_t itn0 = 0, kcn0 = 0, itn1 = 0, kcn1 = 0;   // items and key tiles consumed per slot
+        int st0 = kNeedItem, j0 = 0, n0 = 0, st1 = kNeedItem, j1 = 0, n1 = 0;
+#define PP_INDEP_STEP(T, ITN_, KCN_, ST_, J_, NT_)                                                      \
+  [&]() -> bool {                                                                                       \
+    if (ST_ == kNeedPV) {                                                                               \
+      /* the previous item's epilogue must have read O_T before it is overwritten */                    \
+      if (J_ == 0 && !mbar_try_wait(bar_o_empty + 8 * T, (ITN_ & 1u) ^ 1u)) return false;               \
+      if (!mbar_try_wait(bar_p_full + 8 * T, KCN_ & 1u)) return false;                                  \
+      if (!mbar_try_wait(bar_v_full + 8 * T, KCN_ & 1u)) return false;                                  \
+      tc_fence_after(); /* O_T (+)= P_T V_j */                                                          \
+      const uint32_t a = tmem_base + Cfg::kTmemS + 128u * T;                                            \
+      const uint32_t d = tmem_base + Cfg::kTmemO + (uint32_t)D * T;                                     \
+      const uint32_t b_lo = v_lo0 + (uint32_t)T * (Cfg::kKVBytes >> 4);                                 \
+      mma_ts(d, a, b_lo, idesc_pv, J_ == 0 ? 0u : 1u);                                                  \
+      _Pragma("unroll") for (int kk = 1; kk < BN / 16; ++kk)                                            \
+        mma_ts(d, a + kk * 8, b_lo + (uint32_t)kk * ((16 * 128) >> 4), idesc_pv, 1u);                   \
+      tc_commit(bar_v_empty + 8 * T);                                                                   \
+      ++KCN_;                                                                                           \
+      if (++J_ == NT_) {                                                                                \
+        tc_commit(bar_o_full + 8 * T);                                                                  \
+        ++ITN_;                                                                                         \
+        ST_ = kNeedItem;                                                                                \
+      } else {                                                                                          \
+        ST_ = kNeedS;                                                                                   \
+      }                                                                                                 \
+      return true;                                                                                      \
+    }                                                                                                   \
+    if (ST_ == kNeedS) {                                                                                \
+      if (J_ == 0 && !mbar_try_wait(bar_q_full + 8 * T, ITN_ & 1u)) return false;                       \
+      if (!mbar_try_wait(bar_k_full + 8 * T, KCN_ & 1u)) return false;                                  \
+      tc_fence_after(); /* S_T = Q_T K_j^T */                                                           \
+      const uint32_t d = tmem_base + Cfg::kTmemS + 128u * T;                                            \
+      const uint32_t a_lo = q_lo0 + (uint32_t)T * (Cfg::kQBytes >> 4);                                  \
+      const uint32_t b_lo = k_lo0 + (uint32_t)T * (Cfg::kKVBytes >> 4);                                 \
+      _Pragma("unroll") for (int kk = 0; kk < D / 16; ++kk) {                                           \
+        constexpr uint32_t kChunkQ = (BM * 128) >> 4, kChunkK = (BN * 128) >> 4;                        \
+        mma_ss(d, a_lo + (uint32_t)(kk >> 2) * kChunkQ + (uint32_t)(kk & 3) * 2,                        \
+               b_lo + (uint32_t)(kk >> 2) * kChunkK + (uint32_t)(kk & 3) * 2, idesc_qk,                 \
+               kk > 0 ? 1u : 0u);                                                                       \
+      }                                                                                                 \
+      tc_commit(bar_k_empty + 8 * T);                                                                   \
+      tc_commit(bar_s_full + 8 * T);                                                                    \
+      if (J_ + 1 == NT_) tc_commit(bar_q_empty + 8 * T); /* last read of Q_T in this item */            \
+      ST_ = kNeedPV;                                                                                    \
+      return true;                                                                                      \
+    }                                                                                                   \
+    if (ST_ == kNeedItem) {                                                                             \
+      const uint32_t ring = ITN_ % kRing;                                                               \
+      if (!mbar_try_wait(bar_item_full + 8 * (T * kRing + ring), (ITN_ / kRing) & 1u)) return false;    \
+      const volatile int* e = s_ring + (T * (int)kRing + (int)ring) * kRingInts;                        \
+      const int w = e[0];                                                                               \
+      NT_ = e[3];                                                                                       \
+      mbar_arrive(bar_item_empty + 8 * (T * kRing + ring));                                             \
+      if (w < 0) { ST_ = kDone; return true; }                                                          \
+      J_ = 0;                                                                                           \
+      ST_ = kNeedS;                                                                                     \
+      return true;                                                                                      \
+    }                                                                                                   \
+    return false;                                                                                       \
+  }()
+        unsigned long long idle_since = 0;
+        uint32_t idle_spins = 0;
+        while (st0 != kDone || st1 != kDone) {
+          const bool a0 = PP_INDEP_STEP(0, itn0, kcn0, st0, j0, n0);
+          const bool a1 = PP_INDEP_STEP(1, itn1, kcn1, st1, j1, n1);
+          if (a0 || a1) { idle_spins = 0; continue; }
+          if (idle_spins++ == 0) idle_since = global_ns();
+          if ((idle_spins & 255u) == 0) {           // bounded: give up like every other wait
+            if (*s_abort) break;
+            if (global_ns() - idle_since > wctx.limit_ns) {
+              *s_abort = 1;
+              if (wctx.status) atomicCAS(wctx.status, 0, (int)kWaitP);
+              break;
+            }
+          }
+        }
+#undef PP_INDEP_STEP
+      }
+    } else {
     if (warp == 0 && lane == 0) {
       // ---------------------------------------------------------------- work fetch + K/V producer
       uint32_t it_n = 0, kc = 0;
@@ -573,6 +714,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       PROF_STORE(0, 8);
     }
+    }   // shared-stream roles
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
@@ -595,7 +737,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     bool ok = true;
     PROF_DECL(12);
     while (true) {
-      const uint32_t ring = it_n % kRing;
+      // in independent mode slot t has its own ring, and an item describes one tile (its slot-0 fields)
+      const uint32_t ring = (kIndep ? (uint32_t)t * kRing : 0u) + it_n % kRing;
+      const int f = kIndep ? 0 : t;                    // which slot fields of the entry to read
       PROF_LAP(8);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull));
       PROF_LAP(0);
@@ -603,10 +747,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const volatile int* e = s_ring + ring * kRingInts;
       const int w = e[0];
       const int item_bin = e[1], item_kv_row0 = e[2];
-      const int jb_t = t ? e[6] : 0, je_t = t ? e[8] : e[7];
-      const int q_row0_t = e[4 + t], head_t = e[9 + t];
-      const int bin_used = e[12], seg_end = e[13], key_lo_t = e[14 + t], seg_first_t = e[16 + t];
-      const int single_seg = e[18];
+      const int jb_t = f ? e[6] : 0, je_t = f ? e[8] : e[7];
+      const int q_row0_t = e[4 + f], head_t = e[9 + f];
+      const int bin_used = e[12], seg_end = e[13], key_lo_t = e[14 + f], seg_first_t = e[16 + f];
+      const int single_seg = e[18] >> f;
       mbar_arrive(bar_item_empty + 8 * ring);
       if (w < 0) break;
       const bool used = jb_t < je_t;
@@ -614,7 +758,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       int key_lo = 1, key_hi = 0;                      // visible keys [key_lo, key_hi]; empty for padding
       if (used && i_row < bin_used) {
         key_lo = key_lo_t;
-        if (!((single_seg >> t) & 1)) {                // several prompts in this tile: walk their starts
+        if (!(single_seg & 1)) {                       // several prompts in this tile: walk their starts
           for (int sg = seg_first_t + 1; sg < seg_end; ++sg) {
             const int st = __ldg(tb + args.off_seg_start + sg);
             if (st > i_row) break;
@@ -872,7 +1016,7 @@ int sm_count() {
   return cached;
 }
 
-template <int D>
+template <int D, bool kIndep>
 int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
                        const void* k, const void* v, void* o, int32_t* device_status, cudaStream_t stream) {
   using Cfg = AttnCfg<D>;
@@ -884,7 +1028,7 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
   static bool configured = false;   // per process, per template instance
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<D, kIndep>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Cfg::kSmemBytes);
     if (e != cudaSuccess) return note_cuda_error((int)e, "cudaFuncSetAttribute(smem)");
     configured = true;
@@ -900,7 +1044,7 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   a.off_items = L.items;
   a.n_items = L.n_items;
   a.group = p.n_q_heads / p.n_kv_heads;
-  a.pair_heads = (a.group % 2 == 0) ? 1 : 0;
+  a.pair_heads = (!kIndep && a.group % 2 == 0) ? 1 : 0;
   a.subs = a.pair_heads ? a.group / 2 : a.group;
   a.n_q_heads = p.n_q_heads;
   a.capacity = p.capacity;
@@ -913,7 +1057,7 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   a.status = device_status;
   a.wait_limit_ns = wait_limit_ns();
   const unsigned grid = (unsigned)(total < sms ? total : sms);
-  attention_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, mo, a);
+  attention_kernel<D, kIndep><<<grid, kAttnThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, mo, a);
   const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "attention kernel launch");
 }
@@ -929,8 +1073,12 @@ extern "C" int pp_debug_read_profile(long long* host, int n) {
 int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
                      const void* k, const void* v, void* o, int32_t* device_status, void* stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (p.head_dim == 128) return launch_attention_t<128>(p, d_table, L, q, k, v, o, device_status, s);
-  return launch_attention_t<64>(p, d_table, L, q, k, v, o, device_status, s);
+  if (L.independent_slots) {
+    if (p.head_dim == 128) return launch_attention_t<128, true>(p, d_table, L, q, k, v, o, device_status, s);
+    return launch_attention_t<64, true>(p, d_table, L, q, k, v, o, device_status, s);
+  }
+  if (p.head_dim == 128) return launch_attention_t<128, false>(p, d_table, L, q, k, v, o, device_status, s);
+  return launch_attention_t<64, false>(p, d_table, L, q, k, v, o, device_status, s);
 }
 
 }  // namespace pp

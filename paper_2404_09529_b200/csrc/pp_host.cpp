@@ -180,9 +180,38 @@ size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k) {
   return (size_t)(kHeaderInts + up4(n_bins + 1) + up4(n_bins) + up4(k) + kItemInts * q_tiles);
 }
 
+namespace {
+// Mean key tiles per 128-row query tile of the packing: the measure of how long work items are.
+double mean_key_tiles(int32_t n_bins, const int32_t* bin_seg_ptr, const int32_t* seg_start,
+                      const int32_t* seg_len) {
+  int64_t q_tiles = 0, kv_tiles = 0;
+  for (int32_t b = 0; b < n_bins; ++b) {
+    const int32_t s_lo = bin_seg_ptr[b], s_hi = bin_seg_ptr[b + 1];
+    const int32_t used = seg_start[s_hi - 1] + seg_len[s_hi - 1];
+    int32_t s = s_lo;
+    for (int32_t q0 = 0; q0 < used; q0 += kTileM) {
+      while (s + 1 < s_hi && seg_start[s + 1] <= q0) ++s;
+      const int32_t kv_lo = (seg_start[s] / kTileN) * kTileN;
+      kv_tiles += (std::min(q0 + kTileM, used) - kv_lo + kTileN - 1) / kTileN;
+      ++q_tiles;
+    }
+  }
+  return q_tiles ? (double)kv_tiles / (double)q_tiles : 0.0;
+}
+}  // namespace
+
 int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
-                         const int32_t* seg_start, const int32_t* seg_len, int32_t k, bool pair_rows,
+                         const int32_t* seg_start, const int32_t* seg_len, int32_t k, int32_t group,
                          int32_t* out, size_t out_ints, TableLayout* layout) {
+  // How the two query-tile slots of a CTA are fed:
+  //  - even number of query heads per KV head: two heads over the same rows share a K/V stream;
+  //  - otherwise, long items: two consecutive row tiles of one head share a K/V stream (halves the
+  //    K/V traffic from L2, which long sequences need);
+  //  - otherwise, short items: every slot draws its own single-tile items (a pair of row tiles
+  //    of different length would leave one slot idle for a tile per item).
+  const bool even_group = (group % 2) == 0;
+  const bool independent = !even_group && mean_key_tiles(n_bins, bin_seg_ptr, seg_start, seg_len) < 8.0;
+  const bool pair_rows = !even_group && !independent;
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
   TableLayout L;
   L.bin_seg_ptr = kHeaderInts;
@@ -268,6 +297,7 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   out[9] = (int32_t)std::min<int64_t>(tiles, INT32_MAX);
   out[kHeaderCounter] = 0;   // work counter the CTAs draw from; reset by every upload
   L.total_ints = (int32_t)(L.items + kItemInts * (int64_t)items.size());
+  L.independent_slots = independent;
   if (layout) *layout = L;
   return PP_OK;
 }

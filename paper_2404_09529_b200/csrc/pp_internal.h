@@ -41,13 +41,14 @@ struct TableLayout {
   int32_t items = 0;        // [n_items] WorkItem, longest first
   int32_t n_items = 0;
   int32_t total_ints = 0;
+  bool independent_slots = false;   // items are single tiles, drawn by each slot on its own
 };
 
 int validate_packing(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
                      const int32_t* seg_start, const int32_t* seg_len, int32_t k);
 size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k);
 int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
-                         const int32_t* seg_start, const int32_t* seg_len, int32_t k, bool pair_rows,
+                         const int32_t* seg_start, const int32_t* seg_len, int32_t k, int32_t group,
                          int32_t* out, size_t out_ints, TableLayout* layout);
 
 // Records a failed CUDA call for pp_last_cuda_error(); returns PP_ERR_CUDA.
