@@ -127,6 +127,21 @@ def workload_counts(cfg, lengths):
         unpack_bytes=8 * total * d * hkv)                      # read K', V; write both caches
 
 
+def max_over_ranks(ms: float, dist=None, device="cpu") -> float:
+    """Slowest rank's time: the timed region of a multi-rank run ends when the last rank does."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, tokens_per_rank: int, ms_per_step: float) -> float:
+    """Replicas only: every rank prefills its own copy of the batch, no data-path collective."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def time_loop(fn, iters, warmup=3):
     import torch
     for _ in range(warmup):
@@ -270,12 +285,9 @@ def main():
     clocks = sampler.stop()
     if batch.device_status() != 0:
         raise SystemExit("device-side wait gave up during the timed region")
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = world * T / (ms_per_step * 1e-3)
+    value = whole_job_tokens_per_s(world, T, ms_per_step)
 
     # ---------------------------------------------------------------- per-kernel times (rank-local)
     n_it = args.kernel_iters
@@ -343,13 +355,10 @@ def main():
     e1.record()
     barrier()
     ms_e2e = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e = max_over_ranks(ms_e2e, dist, "cuda")
     h2d = (hq.numel() + hk.numel() + hv.numel()) * 2
     d2h = (ho.numel() + hkc.numel() + hvc.numel()) * 2
-    e2e = {"value": world * T / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": whole_job_tokens_per_s(world, T, ms_e2e / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
            "api": "pp_prefill_host (pinned host buffers, one H2D copy per prompt and tensor)"}
 

@@ -142,6 +142,16 @@ int pp_prefill_attention(const pp_attn_params* params,
                          void* workspace, void* host_workspace, size_t workspace_bytes,
                          int32_t* device_status, void* stream);
 
+/*
+ * Self-test of the kernels' bounded waits (every mbarrier wait inside pp_prefill_attention gives up
+ * after a time limit instead of spinning forever). Enqueues a one-block kernel in which a thread
+ * waits on a barrier that nothing signals; after limit_ms (1..1000) the wait gives up and writes
+ * the non-zero code 77 to *device_status (device int32, zeroed by the caller), and the kernel
+ * returns normally. No counterpart in the paper. Errors: PP_ERR_INVALID_ARG, PP_ERR_UNSUPPORTED,
+ * PP_ERR_CUDA.
+ */
+int pp_selftest_bounded_wait(int32_t* device_status, uint32_t limit_ms, void* stream);
+
 /* Bytes of workspace pp_unpack_kv needs for k prompts (device and host staging alike). */
 size_t pp_unpack_workspace_bytes(int32_t k);
 

@@ -57,6 +57,7 @@ def load_library():
         "pp_prefill_workspace_bytes": (ctypes.c_size_t, [pp, ctypes.c_int32]),
         "pp_prefill_attention": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp,
                                                 ctypes.c_size_t, vp, vp]),
+        "pp_selftest_bounded_wait": (ctypes.c_int, [vp, ctypes.c_uint32, vp]),
         "pp_unpack_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32]),
         "pp_unpack_kv": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, i64p, i32p, vp, vp,
                                         ctypes.c_size_t, vp]),
@@ -152,6 +153,11 @@ def pp_fill_position_ids(pack: Packing):
 
 def pp_prefill_workspace_bytes(params: AttnParams, k: int) -> int:
     return int(load_library().pp_prefill_workspace_bytes(ctypes.byref(params), k))
+
+
+def pp_selftest_bounded_wait(device_status, limit_ms: int, stream: int = 0) -> None:
+    _check(load_library().pp_selftest_bounded_wait(_addr(device_status), limit_ms, stream),
+           "pp_selftest_bounded_wait")
 
 
 def pp_unpack_workspace_bytes(k: int) -> int:

@@ -101,6 +101,13 @@ extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t*
   return PP_OK;
 }
 
+extern "C" int pp_selftest_bounded_wait(int32_t* device_status, uint32_t limit_ms, void* stream) {
+  if (!device_status || limit_ms == 0 || limit_ms > 1000) return PP_ERR_INVALID_ARG;
+  int st = pp::check_device();
+  if (st != PP_OK) return st;
+  return pp::launch_bounded_wait_selftest(device_status, (uint64_t)limit_ms * 1000000ull, stream);
+}
+
 extern "C" size_t pp_unpack_workspace_bytes(int32_t k) { return pp::unpack_table_bytes(k); }
 
 extern "C" int pp_unpack_kv(const pp_attn_params* params, const int32_t* bin_of, const int32_t* off_of,

@@ -965,6 +965,23 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   }
 }
 
+// Self-test of the bounded-wait mechanism: one thread waits on an mbarrier that nothing ever
+// arrives on. The wait must give up after `limit_ns`, write its code to the status word and let
+// the kernel return normally.
+__global__ void bounded_wait_selftest_kernel(int32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const WaitCtx wctx{&abort_flag, status, limit_ns};
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, wctx, 77);
+  __syncthreads();
+}
+
 // ------------------------------------------------------------------------------------------
 // Host side: tensor maps and launch
 // ------------------------------------------------------------------------------------------
@@ -1063,6 +1080,12 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
 }
 
 }  // namespace
+
+int launch_bounded_wait_selftest(int32_t* device_status, uint64_t limit_ns, void* stream) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(device_status, limit_ns);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "self-test kernel launch");
+}
 
 #ifdef PP_PROFILE
 extern "C" int pp_debug_read_profile(long long* host, int n) {

@@ -210,7 +210,7 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   //  - otherwise, short items: every slot draws its own single-tile items (a pair of row tiles
   //    of different length would leave one slot idle for a tile per item).
   const bool even_group = (group % 2) == 0;
-  const bool independent = !even_group && mean_key_tiles(n_bins, bin_seg_ptr, seg_start, seg_len) < 8.0;
+  const bool independent = mean_key_tiles(n_bins, bin_seg_ptr, seg_start, seg_len) < 8.0;
   const bool pair_rows = !even_group && !independent;
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
   TableLayout L;

@@ -63,6 +63,8 @@ int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayou
 int launch_unpack(const pp_attn_params& p, const int32_t* d_table, int32_t k, int64_t total_tokens,
                   const void* k_rot, const void* v, void* k_cache, void* v_cache, void* stream);
 
+int launch_bounded_wait_selftest(int32_t* device_status, uint64_t limit_ns, void* stream);
+
 // Unpack table (int32 units): header 4 ints, then token_prefix[k+1], bin_of[k], off_of[k],
 // cache_cap[k], cache_off as int64[k] (8-byte aligned).
 size_t unpack_table_bytes(int32_t k);

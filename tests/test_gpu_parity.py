@@ -160,3 +160,20 @@ def test_host_buffer_entry_point_matches_device_path():
     assert (params.n_bins, params.capacity) == (4, 112)
     assert torch.equal(o, ref.o_tokens().cpu())
     assert torch.equal(kc, ref.k_cache.cpu()) and torch.equal(vc, ref.v_cache.cpu())
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A device-side wait that nothing satisfies returns a status instead of hanging; the context
+    stays usable afterwards."""
+    import time
+    import paper_2404_09529_b200 as pp
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = time.time()
+    pp.pp_selftest_bounded_wait(status, 5, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 2.0
+    assert int(status.item()) == 77
+    # the device still works: run the tiny workload right after
+    cfg, lengths, q, k, v = _workload("tiny")
+    batch = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    compare_full(batch, lengths, q, k, v, cfg.rope_base)
