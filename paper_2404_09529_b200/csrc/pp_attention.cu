@@ -729,8 +729,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t tmem_o = tmem_base + Cfg::kTmemO + (uint32_t)D * t + lane_base;
     volatile float* x_mine = s_xchg + (t * 2 + h) * 128 + row;
     volatile float* x_other = s_xchg + (t * 2 + (h ^ 1)) * 128 + row;
-    const int bar_slot = 1 + t;                      // named barrier of the slot's 256 threads
-    const int bar_epi = 3 + t;                       // named barrier of the slot's 128 half-0 threads
+    const int bar_pair = 1 + t * 4 + quad;           // named barrier of the two warps that share these rows
+    const int bar_epi = 9 + t;                       // named barrier of the slot's 128 half-0 threads
     const float c_scale = args.scale_log2;
     const int32_t* tb = args.table;
     uint32_t it_n = 0, tcount = 0;
@@ -833,7 +833,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // Row maximum over both halves. The barrier also orders the two halves' S reads before
         // either writes P over the S columns.
         *x_mine = mx;
-        asm volatile("bar.sync %0, %1;" ::"r"(bar_slot), "n"(kSoftmaxThreads) : "memory");
+        asm volatile("bar.sync %0, 64;" ::"r"(bar_pair) : "memory");
         mx = fmaxf(mx, *x_other);
         PROF_LAP(3);
         // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
@@ -906,9 +906,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // the half-1 threads hand their share of the row sum to the half-0 threads, which run the
         // epilogue; the second barrier keeps the exchange slot from being reused too early
         if (h == 1) *x_mine = l_run;
-        asm volatile("bar.sync %0, %1;" ::"r"(bar_slot), "n"(kSoftmaxThreads) : "memory");
+        asm volatile("bar.sync %0, 64;" ::"r"(bar_pair) : "memory");
         const float l_row = (h == 0) ? l_run + *x_other : 0.f;
-        asm volatile("bar.sync %0, %1;" ::"r"(bar_slot), "n"(kSoftmaxThreads) : "memory");
+        asm volatile("bar.sync %0, 64;" ::"r"(bar_pair) : "memory");
         if (h == 0) {
           tc_fence_after();
           const float inv_l = l_row > 0.f ? 1.f / l_row : 0.f;
