@@ -57,6 +57,9 @@ def load_library():
         "pp_prefill_workspace_bytes": (ctypes.c_size_t, [pp, ctypes.c_int32]),
         "pp_prefill_attention": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp,
                                                 ctypes.c_size_t, vp, vp]),
+        "pp_prefill_fused_workspace_bytes": (ctypes.c_size_t, [pp, ctypes.c_int32]),
+        "pp_prefill_fused": (ctypes.c_int, [pp, i32p, i32p, i32p, i32p, ctypes.c_int32, i32p, vp, vp, vp, vp, vp, vp,
+                                            i64p, i32p, vp, vp, ctypes.c_size_t, vp, vp]),
         "pp_selftest_bounded_wait": (ctypes.c_int, [vp, ctypes.c_uint32, vp]),
         "pp_unpack_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32]),
         "pp_unpack_kv": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, i64p, i32p, vp, vp,
@@ -155,6 +158,23 @@ def pp_prefill_workspace_bytes(params: AttnParams, k: int) -> int:
     return int(load_library().pp_prefill_workspace_bytes(ctypes.byref(params), k))
 
 
+def pp_prefill_fused_workspace_bytes(params: AttnParams, k: int) -> int:
+    return int(load_library().pp_prefill_fused_workspace_bytes(ctypes.byref(params), k))
+
+
+def pp_prefill_fused(params: AttnParams, pack: Packing, lengths, q, k, v, o, k_cache, v_cache, cache_off,
+                     cache_cap, workspace, host_workspace, workspace_bytes: int, device_status=None,
+                     stream: int = 0) -> None:
+    l, cc = _i32(lengths), _i32(cache_cap)
+    co = np.ascontiguousarray(np.asarray(cache_off, dtype=np.int64))
+    st = load_library().pp_prefill_fused(
+        ctypes.byref(params), _p32(pack.bin_seg_ptr), _p32(pack.seg_start), _p32(pack.seg_len),
+        _p32(pack.seg_prompt), pack.k, _p32(l), _addr(q), _addr(k), _addr(v), _addr(o), _addr(k_cache),
+        _addr(v_cache), co.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), _p32(cc), _addr(workspace),
+        _addr(host_workspace), workspace_bytes, _addr(device_status), stream)
+    _check(st, "pp_prefill_fused")
+
+
 def pp_selftest_bounded_wait(device_status, limit_ms: int, stream: int = 0) -> None:
     _check(load_library().pp_selftest_bounded_wait(_addr(device_status), limit_ms, stream),
            "pp_selftest_bounded_wait")
@@ -226,9 +246,13 @@ class Workspaces:
         self.unpack_bytes = pp_unpack_workspace_bytes(k)
         if self.attn_bytes == 0 or self.unpack_bytes == 0:
             raise PrepackError(-1, "Workspaces")
+        self.fused_bytes = pp_prefill_fused_workspace_bytes(params, k)
+        self.fused_dev = torch.empty(self.fused_bytes, dtype=torch.uint8, device=device)
         self.attn_dev = torch.empty(self.attn_bytes, dtype=torch.uint8, device=device)
         self.unpack_dev = torch.empty(self.unpack_bytes, dtype=torch.uint8, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self._fused_host = [torch.empty(self.attn_bytes + 32 * k + 256, dtype=torch.uint8).pin_memory()
+                            for _ in range(ring)]
         self._ring = [(torch.empty(self.attn_bytes, dtype=torch.uint8).pin_memory(),
                        torch.empty(self.unpack_bytes, dtype=torch.uint8).pin_memory(),
                        torch.cuda.Event()) for _ in range(ring)]
@@ -243,6 +267,9 @@ class Workspaces:
         if self._used[i]:
             ev.synchronize()
         return a, u, i
+
+    def fused_host(self, slot: int):
+        return self._fused_host[slot]
 
     def release(self, slot: int, stream=None) -> None:
         """Record, on the stream the copies were enqueued on, that slot's buffers may be reused after it."""

@@ -95,10 +95,90 @@ extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t*
     if (st != PP_OK) return st;
   }
   if (do_attn) {
-    st = pp::launch_attention(*params, d_table, L, q, k_, v, o, device_status, stream);
+    st = pp::launch_attention(*params, d_table, L, q, k_, v, o, nullptr, device_status, stream);
     if (st != PP_OK) return st;
   }
   return PP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Fused path: rotation of K + UNPACK in one pass, Q rotated inside the attention kernel
+// ------------------------------------------------------------------------------------------
+namespace pp {
+namespace {
+struct FusedLayout {
+  size_t table_ints;      // prefill table (segment table + work list)
+  size_t off_true_len, off_cap, off_cache_off;   // int32 offsets of the per-segment arrays
+  size_t upload_ints;     // ints copied from the host staging buffer
+  size_t off_rope_bytes;  // byte offset of the cos/sin table (device only)
+  size_t total_bytes;
+};
+FusedLayout fused_layout(const pp_attn_params& p, int32_t k) {
+  auto up4 = [](size_t x) { return (x + 3) & ~size_t(3); };
+  FusedLayout f;
+  f.table_ints = prefill_table_ints(p.n_bins, p.capacity, k);
+  f.off_true_len = up4(f.table_ints);
+  f.off_cap = f.off_true_len + up4((size_t)k);
+  f.off_cache_off = f.off_cap + up4((size_t)k);          // multiple of 4 ints: 16-byte aligned int64 data
+  f.upload_ints = f.off_cache_off + 2 * (size_t)k;
+  f.off_rope_bytes = (f.upload_ints * sizeof(int32_t) + 255) & ~size_t(255);
+  f.total_bytes = f.off_rope_bytes + (size_t)p.capacity * (p.head_dim / 2) * sizeof(float) * 2;
+  return f;
+}
+}  // namespace
+}  // namespace pp
+
+extern "C" size_t pp_prefill_fused_workspace_bytes(const pp_attn_params* params, int32_t k) {
+  if (pp::check_params(params) != PP_OK || k < 1) return 0;
+  return pp::fused_layout(*params, k).total_bytes;
+}
+
+extern "C" int pp_prefill_fused(const pp_attn_params* params, const int32_t* bin_seg_ptr,
+                                const int32_t* seg_start, const int32_t* seg_len, const int32_t* seg_prompt,
+                                int32_t k, const int32_t* lengths, const void* q, void* k_, const void* v, void* o,
+                                void* k_cache, void* v_cache, const int64_t* cache_off, const int32_t* cache_cap,
+                                void* workspace, void* host_workspace, size_t workspace_bytes,
+                                int32_t* device_status, void* stream) {
+  int st = pp::check_params(params);
+  if (st != PP_OK) return st;
+  if (!q || !k_ || !v || !o || !k_cache || !v_cache || !cache_off || !cache_cap || !seg_prompt || !lengths ||
+      !workspace || !host_workspace)
+    return PP_ERR_INVALID_ARG;
+  st = pp::validate_packing(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k);
+  if (st != PP_OK) return st;
+  if (!pp::aligned16(q) || !pp::aligned16(k_) || !pp::aligned16(v) || !pp::aligned16(o) ||
+      !pp::aligned16(k_cache) || !pp::aligned16(v_cache) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return PP_ERR_ALIGNMENT;
+  const pp::FusedLayout f = pp::fused_layout(*params, k);
+  if (workspace_bytes < f.total_bytes) return PP_ERR_BUFFER_TOO_SMALL;
+  int32_t* h = static_cast<int32_t*>(host_workspace);
+  int64_t* h_coff = reinterpret_cast<int64_t*>(h + f.off_cache_off);
+  for (int32_t s = 0; s < k; ++s) {
+    const int32_t i = seg_prompt[s];
+    if (i < 0 || i >= k) return PP_ERR_INVALID_ARG;
+    if (lengths[i] < 1 || lengths[i] > seg_len[s] || cache_cap[i] < lengths[i]) return PP_ERR_LENGTH;
+    if (cache_off[i] < 0) return PP_ERR_INVALID_ARG;
+    if (cache_off[i] % 8 != 0) return PP_ERR_ALIGNMENT;
+    h[f.off_true_len + s] = lengths[i];
+    h[f.off_cap + s] = cache_cap[i];
+    h_coff[s] = cache_off[i];
+  }
+  if ((st = pp::check_device()) != PP_OK) return st;
+  pp::TableLayout L;
+  st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
+                                params->n_q_heads / params->n_kv_heads, h, f.table_ints, &L);
+  if (st != PP_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * f.upload_ints,
+                                  cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
+  int32_t* d_table = static_cast<int32_t*>(workspace);
+  void* rope_table = static_cast<char*>(workspace) + f.off_rope_bytes;
+  if ((st = pp::launch_rope_table(*params, rope_table, stream)) != PP_OK) return st;
+  st = pp::launch_rope_unpack(*params, d_table, L, (int32_t)f.off_true_len, (int32_t)f.off_cap,
+                              (int32_t)f.off_cache_off, rope_table, k_, v, k_cache, v_cache, stream);
+  if (st != PP_OK) return st;
+  return pp::launch_attention(*params, d_table, L, q, k_, v, o, rope_table, device_status, stream);
 }
 
 extern "C" int pp_selftest_bounded_wait(int32_t* device_status, uint32_t limit_ms, void* stream) {

@@ -284,6 +284,7 @@ struct AttnArgs {
   int32_t total_work;            // n_kv_heads * n_items * subs
   float scale_log2;              // softmax scale * log2(e)
   __nv_bfloat16* o;
+  const float2* rope_table;      // [capacity][D/2] (cos, sin), or null: Q arrives already rotated
   int32_t* status;
   unsigned long long wait_limit_ns;
 };
@@ -376,6 +377,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const uint32_t bar_v_full = s_misc + 288;      // [4]
   const uint32_t bar_v_empty = s_misc + 320;     // [4]
   volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 352);   // [2 rings][kRing][kRingInts]
+  const uint32_t bar_q_rot = s_misc + 1000;      // [2] Q_t has been rotated in place (fused path)
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 992);
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 996);
   volatile float* s_xchg = reinterpret_cast<volatile float*>(misc + 1024);   // [2 slots][2 halves][128 rows]
@@ -396,6 +398,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_q_full + 8 * i, 1);
       mbar_init(bar_q_empty + 8 * i, 1);
+      mbar_init(bar_q_rot + 8 * i, kSoftmaxThreads);
       mbar_init(bar_s_full + 8 * i, 1);
       mbar_init(bar_p_full + 8 * i, kSoftmaxThreads);
       mbar_init(bar_o_full + 8 * i, 1);
@@ -472,6 +475,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         constexpr uint32_t idesc_qk = instr_desc(BN, false);
         constexpr uint32_t idesc_pv = instr_desc(D, true);
         const uint32_t q_lo0 = desc_lo(s_q, 0), k_lo0 = desc_lo(s_k, 0), v_lo0 = desc_lo(s_v, BN * 128);
+        const uint32_t bar_q_ready = args.rope_table ? bar_q_rot : bar_q_full;
         enum { kNeedItem = 0, kNeedS, kNeedPV, kDone };
         uint32_t itn0 = 0, kcn0 = 0, itn1 = 0, kcn1 = 0;   // items and key tiles consumed per slot
         int st0 = kNeedItem, j0 = 0, n0 = 0, st1 = kNeedItem, j1 = 0, n1 = 0;
@@ -501,7 +505,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       return true;                                                                                      \
     }                                                                                                   \
     if (ST_ == kNeedS) {                                                                                \
-      if (J_ == 0 && !mbar_try_wait(bar_q_full + 8 * T, ITN_ & 1u)) return false;                       \
+      if (J_ == 0 && !mbar_try_wait(bar_q_ready + 8 * T, ITN_ & 1u)) return false;                      \
       if (!mbar_try_wait(bar_k_full + 8 * T, KCN_ & 1u)) return false;                                  \
       tc_fence_after(); /* S_T = Q_T K_j^T */                                                           \
       const uint32_t d = tmem_base + Cfg::kTmemS + 128u * T;                                            \
@@ -689,8 +693,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         mbar_arrive(bar_item_empty + 8 * ring);
         if (w < 0) break;
         PROF_LAP(0);
-        ok = mbar_wait(bar_q_full + 0, it_n & 1u, wctx, kWaitQFull) &&
-             mbar_wait(bar_q_full + 8, it_n & 1u, wctx, kWaitQFull);
+        const uint32_t bar_q_ready = args.rope_table ? bar_q_rot : bar_q_full;
+        ok = mbar_wait(bar_q_ready + 0, it_n & 1u, wctx, kWaitQFull) &&
+             mbar_wait(bar_q_ready + 8, it_n & 1u, wctx, kWaitQFull);
         if (!ok) break;
         PROF_LAP(1);
         if (je0 > 0) ok = issue_qk(0, 0);
@@ -766,6 +771,42 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         key_hi = i_row;
+      }
+      if (args.rope_table) {
+        // Fused path: rotate this row's part of the Q tile in shared memory (restart position =
+        // row - start of its prompt), same fp32 arithmetic and rounding as the stand-alone kernel.
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * t, it_n & 1u, wctx, kWaitQFull));
+        if (!ok) break;
+        const int pos = key_hi - key_lo;               // < 0 for padding rows (key_hi = 0, key_lo = 1)
+        if (used && pos > 0) {
+          constexpr int kUnits = D / 16;               // 16-byte units per half of a row
+          const uint32_t q_row = s_q + (uint32_t)t * Cfg::kQBytes + (uint32_t)row * 128;
+          const float4* tab = reinterpret_cast<const float4*>(args.rope_table + (size_t)pos * (D / 2));
+#pragma unroll
+          for (int uu = 0; uu < kUnits / 2; ++uu) {
+            const int u = h * (kUnits / 2) + uu;       // pairs (8u .. 8u+7, + D/2)
+            const uint32_t a_lo = q_row + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4);
+            const uint32_t a_hi = (D == 128)
+                ? q_row + (BM * 128) + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4)
+                : q_row + ((((uint32_t)(u + kUnits)) ^ ((uint32_t)row & 7u)) << 4);
+            uint32_t lo[4], hi[4];
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo[0]), "=r"(lo[1]), "=r"(lo[2]), "=r"(lo[3]) : "r"(a_lo));
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi[0]), "=r"(hi[1]), "=r"(hi[2]), "=r"(hi[3]) : "r"(a_hi));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4 cs = __ldg(tab + u * 4 + i);   // (cos, sin) of two consecutive j
+              const __nv_bfloat162 l2 = *reinterpret_cast<__nv_bfloat162*>(&lo[i]);
+              const __nv_bfloat162 h2 = *reinterpret_cast<__nv_bfloat162*>(&hi[i]);
+              const float2 a = __bfloat1622float2(l2), b = __bfloat1622float2(h2);
+              lo[i] = pack_bf16(__fmaf_rn(a.x, cs.x, -__fmul_rn(b.x, cs.y)), __fmaf_rn(a.y, cs.z, -__fmul_rn(b.y, cs.w)));
+              hi[i] = pack_bf16(__fmaf_rn(b.x, cs.x, __fmul_rn(a.x, cs.y)), __fmaf_rn(b.y, cs.z, __fmul_rn(a.y, cs.w)));
+            }
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_lo), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_hi), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
+        }
+        mbar_arrive(bar_q_rot + 8 * t);
       }
       float m_run = -INFINITY;      // running maximum of the whole row, in scaled log2 units
       float l_run = 0.f;            // this thread's share of the running sum of exp2(s * c - m_run)
@@ -1035,7 +1076,8 @@ int sm_count() {
 
 template <int D, bool kIndep>
 int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
-                       const void* k, const void* v, void* o, int32_t* device_status, cudaStream_t stream) {
+                       const void* k, const void* v, void* o, const void* rope_table, int32_t* device_status,
+                       cudaStream_t stream) {
   using Cfg = AttnCfg<D>;
   CUtensorMap mq, mk, mv, mo;
   int st;
@@ -1071,6 +1113,7 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)D);
   a.scale_log2 = scale * 1.4426950408889634f;
   a.o = static_cast<__nv_bfloat16*>(o);
+  a.rope_table = static_cast<const float2*>(rope_table);
   a.status = device_status;
   a.wait_limit_ns = wait_limit_ns();
   const unsigned grid = (unsigned)(total < sms ? total : sms);
@@ -1094,14 +1137,15 @@ extern "C" int pp_debug_read_profile(long long* host, int n) {
 #endif
 
 int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
-                     const void* k, const void* v, void* o, int32_t* device_status, void* stream) {
+                     const void* k, const void* v, void* o, const void* rope_table, int32_t* device_status,
+                     void* stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (L.independent_slots) {
-    if (p.head_dim == 128) return launch_attention_t<128, true>(p, d_table, L, q, k, v, o, device_status, s);
-    return launch_attention_t<64, true>(p, d_table, L, q, k, v, o, device_status, s);
+    if (p.head_dim == 128) return launch_attention_t<128, true>(p, d_table, L, q, k, v, o, rope_table, device_status, s);
+    return launch_attention_t<64, true>(p, d_table, L, q, k, v, o, rope_table, device_status, s);
   }
-  if (p.head_dim == 128) return launch_attention_t<128, false>(p, d_table, L, q, k, v, o, device_status, s);
-  return launch_attention_t<64, false>(p, d_table, L, q, k, v, o, device_status, s);
+  if (p.head_dim == 128) return launch_attention_t<128, false>(p, d_table, L, q, k, v, o, rope_table, device_status, s);
+  return launch_attention_t<64, false>(p, d_table, L, q, k, v, o, rope_table, device_status, s);
 }
 
 }  // namespace pp

@@ -57,9 +57,18 @@ int note_cuda_error(int cuda_error, const char* what);
 // Kernel launchers (device pointers, stream = cudaStream_t as void*). Return a PP_* status.
 int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
                 void* q, void* k, void* stream);
+// rope_table: device [capacity][D/2] (cos, sin) pairs, or null. When given, q holds the raw
+// queries and the kernel rotates each Q tile in shared memory before use.
 int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayout& L,
-                     const void* q, const void* k, const void* v, void* o,
+                     const void* q, const void* k, const void* v, void* o, const void* rope_table,
                      int32_t* device_status, void* stream);
+// Fused K rotation + UNPACK; the three offsets locate per-segment arrays inside the table
+// (true length, cache capacity: int32; cache element offset: int64).
+int launch_rope_unpack(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
+                       int32_t off_true_len, int32_t off_cap, int32_t off_cache_off, const void* rope_table,
+                       void* k, const void* v, void* k_cache, void* v_cache, void* stream);
+// Fills rope_table for positions 0 .. capacity-1.
+int launch_rope_table(const pp_attn_params& p, void* table, void* stream);
 int launch_unpack(const pp_attn_params& p, const int32_t* d_table, int32_t k, int64_t total_tokens,
                   const void* k_rot, const void* v, void* k_cache, void* v_cache, void* stream);
 

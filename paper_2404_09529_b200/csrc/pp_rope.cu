@@ -35,8 +35,9 @@ __device__ __forceinline__ void rotate8(uint4& lo, uint4& hi, const float* cs, c
     const float2 a = bf2_to_f2(l[i]);
     const float2 b = bf2_to_f2(h[i]);
     const float c0 = cs[2 * i], c1 = cs[2 * i + 1], s0 = sn[2 * i], s1 = sn[2 * i + 1];
-    l[i] = f2_to_bf2(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1);
-    h[i] = f2_to_bf2(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1);
+    // written with explicit fma/mul so that every kernel that rotates gives the same bits
+    l[i] = f2_to_bf2(__fmaf_rn(a.x, c0, -__fmul_rn(b.x, s0)), __fmaf_rn(a.y, c1, -__fmul_rn(b.y, s1)));
+    h[i] = f2_to_bf2(__fmaf_rn(b.x, c0, __fmul_rn(a.x, s0)), __fmaf_rn(b.y, c1, __fmul_rn(a.y, s1)));
   }
 }
 
@@ -114,14 +115,160 @@ rope_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k,
   }
 }
 
-}  // namespace
+// cos/sin of position * theta_j for every position of a bin: table[pos][j] = (cos, sin). Read by
+// the attention kernel, which rotates Q on the fly in the fused path.
+__global__ void __launch_bounds__(256)
+rope_table_kernel(float2* __restrict__ table, int32_t capacity, int32_t half,
+                  const __grid_constant__ RopeFreq freq) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)capacity * half) return;
+  const int32_t pos = (int32_t)(idx / half), j = (int32_t)(idx - (int64_t)pos * half);
+  float sn = 0.f, cs = 1.f;
+  if (pos > 0) {      // same arithmetic as rope_kernel, so both give identical bits
+    const double ang = (double)pos * freq.inv_freq[j];
+    const double n = rint(ang * 0.15915494309189535);
+    double red = fma(-n, 6.283185307179586, ang);
+    red = fma(-n, 2.4492935982947064e-16, red);
+    sincosf((float)red, &sn, &cs);
+  }
+  table[idx] = make_float2(cs, sn);
+}
 
-int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L, void* q,
-                void* k, void* stream) {
+// Fused K rotation + UNPACK (Algorithm 1 lines 7-8 in one pass over K and V): every real packed
+// row of K is rotated (cos/sin from the table), written back to the packed tensor (the attention
+// kernel reads it there) and into its prompt's K cache; the V row is copied into the V cache.
+struct SegExt {                    // per-segment arrays appended to the prefill table
+  int32_t off_true_len, off_cap, off_cache_off;   // int32 offsets into the table (cache_off: int64 data)
+};
+
+template <int D>
+__global__ void __launch_bounds__(kRopeThreads)
+rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                   __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
+                   const int32_t* __restrict__ table, int32_t off_bin_seg_ptr, int32_t off_bin_used,
+                   int32_t off_seg_start, SegExt ext, const float2* __restrict__ rope_table,
+                   int32_t n_bins, int32_t capacity, int32_t n_kv_heads) {
+  constexpr int kHalf = D / 2;
+  constexpr int kPairUnits = kHalf / 8;             // (lower, upper) 16-byte pairs per head
+  constexpr int kVecs = D / 8;                      // 16-byte vectors per head
+  __shared__ int32_t s_pos[kRopeRows];              // restart position, -1 for padding rows
+  __shared__ int64_t s_dst[kRopeRows];              // cache element offset of (head 0, this position); -1: not cached
+  __shared__ int64_t s_head_stride[kRopeRows];      // cache_cap * D
+
+  const int64_t row0 = (int64_t)blockIdx.x * kRopeRows;
+  const int64_t n_rows = (int64_t)n_bins * capacity;
+  const int tid = threadIdx.x;
+  if (tid < kRopeRows) {
+    const int64_t row = row0 + tid;
+    int32_t pos = -1;
+    int64_t dst = -1, stride = 0;
+    if (row < n_rows) {
+      const int32_t b = (int32_t)(row / capacity);
+      const int32_t t = (int32_t)(row - (int64_t)b * capacity);
+      if (t < table[off_bin_used + b]) {
+        int32_t lo = table[off_bin_seg_ptr + b], hi = table[off_bin_seg_ptr + b + 1] - 1;
+        while (lo < hi) {
+          const int32_t mid = (lo + hi + 1) >> 1;
+          if (table[off_seg_start + mid] <= t) lo = mid; else hi = mid - 1;
+        }
+        pos = t - table[off_seg_start + lo];
+        if (pos < table[ext.off_true_len + lo]) {   // rows past the prompt's true length are not cached
+          const int64_t* coff = reinterpret_cast<const int64_t*>(table + ext.off_cache_off);
+          stride = (int64_t)table[ext.off_cap + lo] * D;
+          dst = coff[lo] + (int64_t)pos * D;
+        }
+      }
+    }
+    s_pos[tid] = pos;
+    s_dst[tid] = dst;
+    s_head_stride[tid] = stride;
+  }
+  __syncthreads();
+
+  const int units_k = n_kv_heads * kPairUnits;
+  const int units_v = n_kv_heads * kVecs;
+  const int units_per_row = units_k + units_v;
+  for (int u = tid; u < kRopeRows * units_per_row; u += kRopeThreads) {
+    const int r = u / units_per_row;
+    int w = u - r * units_per_row;
+    const int32_t pos = s_pos[r];
+    if (pos < 0) continue;                          // padding row
+    const int64_t row = row0 + r;
+    const int64_t dst = s_dst[r];
+    if (w < units_k) {
+      const int head = w / kPairUnits, c = w - head * kPairUnits;
+      __nv_bfloat16* base = k + (row * n_kv_heads + head) * D;
+      uint4 lo = *reinterpret_cast<const uint4*>(base + c * 8);
+      uint4 hi = *reinterpret_cast<const uint4*>(base + kHalf + c * 8);
+      if (pos > 0) {
+        float cs[8], sn[8];
+        const float4* tab = reinterpret_cast<const float4*>(rope_table + (size_t)pos * kHalf + c * 8);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 t4 = __ldg(tab + i);
+          cs[2 * i] = t4.x; sn[2 * i] = t4.y; cs[2 * i + 1] = t4.z; sn[2 * i + 1] = t4.w;
+        }
+        rotate8(lo, hi, cs, sn);
+        *reinterpret_cast<uint4*>(base + c * 8) = lo;
+        *reinterpret_cast<uint4*>(base + kHalf + c * 8) = hi;
+      }
+      if (dst >= 0) {
+        __nv_bfloat16* cd = k_cache + dst + head * s_head_stride[r];
+        *reinterpret_cast<uint4*>(cd + c * 8) = lo;
+        *reinterpret_cast<uint4*>(cd + kHalf + c * 8) = hi;
+      }
+    } else if (dst >= 0) {
+      w -= units_k;
+      const int head = w / kVecs, c = w - head * kVecs;
+      const uint4 val = __ldg(reinterpret_cast<const uint4*>(v + (row * n_kv_heads + head) * D + c * 8));
+      *reinterpret_cast<uint4*>(v_cache + dst + head * s_head_stride[r] + c * 8) = val;
+    }
+  }
+}
+
+RopeFreq make_freq(const pp_attn_params& p) {
   RopeFreq freq;
   const int half = p.head_dim / 2;
   for (int j = 0; j < kMaxHalf; ++j)
     freq.inv_freq[j] = j < half ? pow((double)p.rope_base, -2.0 * j / (double)p.head_dim) : 0.0;
+  return freq;
+}
+
+}  // namespace
+
+int launch_rope_table(const pp_attn_params& p, void* table, void* stream) {
+  const RopeFreq freq = make_freq(p);
+  const int half = p.head_dim / 2;
+  const int64_t n = (int64_t)p.capacity * half;
+  rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<float2*>(table), p.capacity, half, freq);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "rope table kernel launch");
+}
+
+int launch_rope_unpack(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
+                       int32_t off_true_len, int32_t off_cap, int32_t off_cache_off, const void* rope_table,
+                       void* k, const void* v, void* k_cache, void* v_cache, void* stream) {
+  const int64_t n_rows = (int64_t)p.n_bins * p.capacity;
+  const unsigned grid = (unsigned)((n_rows + kRopeRows - 1) / kRopeRows);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const SegExt ext{off_true_len, off_cap, off_cache_off};
+  if (p.head_dim == 128) {
+    rope_unpack_kernel<128><<<grid, kRopeThreads, 0, s>>>(
+        (__nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table,
+        L.bin_seg_ptr, L.bin_used, L.seg_start, ext, (const float2*)rope_table, p.n_bins, p.capacity, p.n_kv_heads);
+  } else {
+    rope_unpack_kernel<64><<<grid, kRopeThreads, 0, s>>>(
+        (__nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table,
+        L.bin_seg_ptr, L.bin_used, L.seg_start, ext, (const float2*)rope_table, p.n_bins, p.capacity, p.n_kv_heads);
+  }
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "rope+unpack kernel launch");
+}
+
+int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L, void* q,
+                void* k, void* stream) {
+  const RopeFreq freq = make_freq(p);
   const int64_t n_rows = (int64_t)p.n_bins * p.capacity;
   const unsigned grid = (unsigned)((n_rows + kRopeRows - 1) / kRopeRows);
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -83,6 +83,18 @@ class PrefillBatch:
                            self.ws.unpack_bytes, stream)
         self.ws.release(slot)
 
+    def run_fused(self, repack: bool = False) -> None:
+        """One pass of the hot path through the fused entry point (asynchronous). q is left untouched."""
+        if repack:
+            self._pack()
+        stream = torch.cuda.current_stream().cuda_stream
+        _, _, slot = self.ws.acquire()
+        self.params.flags = 0
+        B.pp_prefill_fused(self.params, self.pack, self.lengths, self.q, self.kk, self.v, self.o, self.k_cache,
+                           self.v_cache, self.cache_off, self.cache_cap, self.ws.fused_dev,
+                           self.ws.fused_host(slot), self.ws.fused_bytes, self.ws.status, stream)
+        self.ws.release(slot)
+
     def run_unpack_only(self) -> None:
         stream = torch.cuda.current_stream().cuda_stream
         _, host_unpack, slot = self.ws.acquire()

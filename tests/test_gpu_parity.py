@@ -177,3 +177,47 @@ def test_bounded_wait_gives_up_and_reports():
     cfg, lengths, q, k, v = _workload("tiny")
     batch = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
     compare_full(batch, lengths, q, k, v, cfg.rope_base)
+
+
+def _run_fused(lengths, q, k, v, hq, hkv, d, base, mode="packed"):
+    from paper_2404_09529_b200.runner import PrefillBatch
+    b = PrefillBatch(lengths, hq, hkv, d, base, mode=mode)
+    b.load(q, k, v)
+    q_before = b.q.clone()
+    b.run_fused()
+    torch.cuda.synchronize()
+    assert b.device_status() == 0
+    assert torch.equal(b.q, q_before)              # the fused path never rewrites q
+    return b
+
+
+@pytest.mark.parametrize("name,mode", [("tiny", "packed"), ("tiny", "padded"), ("llama2_7b", "packed"),
+                                       ("many_short", "packed")])
+def test_fused_entry_point_matches_two_call_path_bit_for_bit(name, mode):
+    cfg, lengths, q, k, v = _workload(name)
+    a = run_cuda(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, mode)
+    b = _run_fused(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, mode)
+    assert torch.equal(a.k_cache, b.k_cache) and torch.equal(a.v_cache, b.v_cache)
+    assert torch.equal(a.kk.view(-1, a.hkv, a.d)[a.token_rows], b.kk.view(-1, b.hkv, b.d)[b.token_rows])
+    assert torch.equal(a.o_tokens(), b.o_tokens())
+
+
+def test_fused_entry_point_parity_against_oracle():
+    cfg, lengths, q, k, v = _workload("tiny")
+    b = _run_fused(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    compare_full(b, lengths, q, k, v, cfg.rope_base)
+    lengths = np.array([700, 300, 250, 150, 90, 5, 5], np.int32)
+    q, k, v = _random_case(lengths, 8, 2, 128, seed=11)
+    for mode in ("packed", "padded"):
+        b = _run_fused(lengths, q, k, v, 8, 2, 128, 500000.0, mode)
+        compare_full(b, lengths, q, k, v, 500000.0)
+
+
+@pytest.mark.parametrize("name", ["llama3_8b_gqa", "long_mix"])
+def test_fused_large_configs_sampled_parity(name):
+    cfg, lengths, q, k, v = _workload(name, device="cuda")
+    b = _run_fused(lengths, q, k, v, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    order = np.argsort(lengths)
+    prompts = sorted(set(int(order[i]) for i in (0, len(order) // 2, -1)))
+    compare_sampled(b, lengths, q.cpu(), k.cpu(), v.cpu(), cfg.rope_base, prompts=prompts,
+                    kv_heads=[0, cfg.n_kv_heads - 1], n_rows=32)
