@@ -266,35 +266,60 @@ def main():
 
     batch = PrefillBatch(lengths, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, mode="packed")
     batch.load(q_tok, k_tok, v_tok)
-    step = lambda: batch.run(repack=True)
+    # The whole path has two public routes through the C ABI: three calls (pp_pack +
+    # pp_prefill_attention + pp_unpack_kv) or two (pp_pack + pp_prefill_fused). Both are timed over the
+    # same K steps; the headline is the faster one (named in config.path), the other is reported beside it.
+    routes = {"three_call": lambda: batch.run(repack=True), "fused": lambda: batch.run_fused(repack=True)}
 
-    # ---------------------------------------------------------------- headline: whole path, device resident
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    sampler = ClockSampler(torch.cuda.current_device())
-    sampler.start()
+    def timed_region(step):
+        batch.load(q_tok, k_tok, v_tok)          # raw Q/K again (the three-call route rotates q in place)
+        for _ in range(max(args.warmup, 3)):
+            step()
+        barrier()
+        sampler = ClockSampler(torch.cuda.current_device())
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        clk = sampler.stop()
+        if batch.device_status() != 0:
+            raise SystemExit("device-side wait gave up during the timed region")
+        return max_over_ranks(ms, dist, "cuda") / args.steps, clk
+
+    route_ms, route_clocks = {}, {}
+    for name, fn in routes.items():
+        route_ms[name], route_clocks[name] = timed_region(fn)
+    path = min(route_ms, key=route_ms.get)
+    if dist is not None:                          # all ranks must agree on the headline route
+        flag = torch.tensor([0 if path == "three_call" else 1], device="cuda")
+        dist.broadcast(flag, src=0)
+        path = "three_call" if int(flag.item()) == 0 else "fused"
+    ms_per_step, clocks = route_ms[path], route_clocks[path]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    ms_total = e0.elapsed_time(e1)
-    clocks = sampler.stop()
-    if batch.device_status() != 0:
-        raise SystemExit("device-side wait gave up during the timed region")
-    ms_total = max_over_ranks(ms_total, dist, "cuda")
-    ms_per_step = ms_total / args.steps
     value = whole_job_tokens_per_s(world, T, ms_per_step)
+    batch.load(q_tok, k_tok, v_tok)
 
     # ---------------------------------------------------------------- per-kernel times (rank-local)
     n_it = args.kernel_iters
     ms_rope = time_loop(lambda: batch.run(flags=pp.PP_FLAG_ROPE_ONLY, unpack=False), n_it)
     ms_attn = time_loop(lambda: batch.run(flags=pp.PP_FLAG_SKIP_ROPE, unpack=False), n_it)
     ms_unpack = time_loop(batch.run_unpack_only, n_it)
+    ms_rope_unpack = time_loop(lambda: batch.run_fused(flags=pp.PP_FLAG_ROPE_ONLY), n_it)
+    ms_attn_fused = time_loop(lambda: batch.run_fused(flags=pp.PP_FLAG_SKIP_ROPE), n_it)
+    fused_k_bytes = 2 * T * cfg.head_dim * cfg.n_kv_heads * 5     # K read, K' and K cache written, V read, V cache written
     kernels = {
+        "rope_unpack_fused": {"ms": ms_rope_unpack, "gbs": fused_k_bytes / ms_rope_unpack * 1e-6,
+                              "frac_hbm": fused_k_bytes / ms_rope_unpack * 1e-6 / peaks["hbm_gbs"]},
+        "attention_fused": {"ms": ms_attn_fused, "tflops": counts["useful_flops"] / ms_attn_fused * 1e-9,
+                            "frac_bf16_peak": counts["useful_flops"] / ms_attn_fused * 1e-9 / peaks["bf16_tflops"],
+                            "frac_bf16_datasheet": counts["useful_flops"] / ms_attn_fused * 1e-9 / 2250.0,
+                            "gbs": counts["attn_bytes"] / ms_attn_fused * 1e-6,
+                            "frac_hbm": counts["attn_bytes"] / ms_attn_fused * 1e-6 / peaks["hbm_gbs"]},
         "rope": {"ms": ms_rope, "gbs": counts["rope_bytes"] / ms_rope * 1e-6,
                  "frac_hbm": counts["rope_bytes"] / ms_rope * 1e-6 / peaks["hbm_gbs"]},
         "attention": {"ms": ms_attn, "tflops": counts["useful_flops"] / ms_attn * 1e-9,
@@ -309,14 +334,16 @@ def main():
     intensity = counts["useful_flops"] / counts["attn_bytes"]
     ridge = peaks["bf16_tflops"] * 1e3 / peaks["hbm_gbs"]
     traffic = NCU_ATTENTION_TRAFFIC_BYTES.get(args.workload)
+    # the attention kernel as launched in the headline route
+    dom = kernels["attention_fused"] if path == "fused" else kernels["attention"]
     if intensity < ridge:
-        roofline = {"kernel": "attention", "bound": "hbm", "achieved": kernels["attention"]["gbs"],
-                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": kernels["attention"]["frac_hbm"],
+        roofline = {"kernel": "attention", "bound": "hbm", "achieved": dom["gbs"],
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dom["frac_hbm"],
                     "traffic": traffic, "peak_source": peaks["source"] + " (burst copy)",
                     "flop_per_byte": intensity, "ridge_flop_per_byte": ridge}
     else:
-        roofline = {"kernel": "attention", "bound": "tensor", "achieved": kernels["attention"]["tflops"],
-                    "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": kernels["attention"]["frac_bf16_peak"],
+        roofline = {"kernel": "attention", "bound": "tensor", "achieved": dom["tflops"],
+                    "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": dom["frac_bf16_peak"],
                     "traffic": traffic, "peak_source": peaks["source"] + " (burst, kernel timed alone)",
                     "flop_per_byte": intensity, "ridge_flop_per_byte": ridge}
 
@@ -326,12 +353,16 @@ def main():
         pb = PrefillBatch(lengths, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, mode="padded")
         pb.load(q_tok, k_tok, v_tok)
         n_pad = max(3, min(args.steps, 30))
-        ms_pad = time_loop(lambda: pb.run(repack=True), n_pad)
-        ms_pad_attn = time_loop(lambda: pb.run(flags=pp.PP_FLAG_SKIP_ROPE, unpack=False), max(3, n_pad // 2))
+        if path == "fused":
+            ms_pad = time_loop(lambda: pb.run_fused(repack=True), n_pad)
+            ms_pad_attn = time_loop(lambda: pb.run_fused(flags=pp.PP_FLAG_SKIP_ROPE), max(3, n_pad // 2))
+        else:
+            ms_pad = time_loop(lambda: pb.run(repack=True), n_pad)
+            ms_pad_attn = time_loop(lambda: pb.run(flags=pp.PP_FLAG_SKIP_ROPE, unpack=False), max(3, n_pad // 2))
         padded = {"tokens_per_s": T / (ms_pad * 1e-3), "ms_per_step": ms_pad, "attention_ms": ms_pad_attn,
                   "rows_computed": int(pb.pack.n_bins) * int(pb.pack.capacity),
                   "speedup_packed_vs_padded": ms_pad / ms_per_step,
-                  "attention_speedup_packed_vs_padded": ms_pad_attn / ms_attn}
+                  "attention_speedup_packed_vs_padded": ms_pad_attn / dom["ms"]}
         del pb
         torch.cuda.empty_cache()
 
@@ -379,13 +410,18 @@ def main():
             "config": {"workload": args.workload, "description": cfg.description, "n_prompts": int(len(lengths)),
                        "total_tokens": T, "n_bins": int(batch.pack.n_bins), "capacity": int(batch.pack.capacity),
                        "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
-                       "rope_base": cfg.rope_base, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "rope_base": cfg.rope_base, "path": path, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                        "l2": f"no flush: each step streams {resident_mb:.0f} MB of tensors, larger than the 126 MB L2"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roofline,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": (3 if path == "three_call" else 4) * args.steps, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "kernels": kernels, "padded": padded,
-            "attention": {"useful_tflops": kernels["attention"]["tflops"],
-                          "frac_bf16_peak_measured": kernels["attention"]["frac_bf16_peak"],
-                          "frac_bf16_peak_datasheet": kernels["attention"]["frac_bf16_datasheet"]},
+            "routes": {"three_call": {"tokens_per_s": whole_job_tokens_per_s(world, T, route_ms["three_call"]),
+                                      "ms_per_step": route_ms["three_call"],
+                                      "api": "pp_pack + pp_prefill_attention + pp_unpack_kv"},
+                       "fused": {"tokens_per_s": whole_job_tokens_per_s(world, T, route_ms["fused"]),
+                                 "ms_per_step": route_ms["fused"], "api": "pp_pack + pp_prefill_fused"}},
+            "attention": {"useful_tflops": dom["tflops"],
+                          "frac_bf16_peak_measured": dom["frac_bf16_peak"],
+                          "frac_bf16_peak_datasheet": dom["frac_bf16_datasheet"]},
             "peaks": peaks,
         }
         print(json.dumps(line))

@@ -284,7 +284,7 @@ struct AttnArgs {
   int32_t total_work;            // n_kv_heads * n_items * subs
   float scale_log2;              // softmax scale * log2(e)
   __nv_bfloat16* o;
-  const float2* rope_table;      // [capacity][D/2] (cos, sin), or null: Q arrives already rotated
+  const float2* rope_table;      // [D/4][capacity][2] (cos, sin) pairs, or null: Q arrives already rotated
   int32_t* status;
   unsigned long long wait_limit_ns;
 };
@@ -741,6 +741,49 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     uint32_t it_n = 0, tcount = 0;
     bool ok = true;
     PROF_DECL(12);
+    // Rotates this thread's part of row `row` of Q_t in shared memory by the angles of position
+    // `pos` (<= 0: nothing to do), with the same fp32 arithmetic and rounding as the stand-alone
+    // kernel, then reports the slot's Q as ready. Waits for the TMA load of Q first.
+    auto rotate_q = [&](const int pos, const uint32_t parity) -> bool {
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * t, parity, wctx, kWaitQFull))) return false;
+      if (pos > 0) {
+        constexpr int kUnits = D / 16;                 // 16-byte units per half of a row
+        const uint32_t q_row = s_q + (uint32_t)t * Cfg::kQBytes + (uint32_t)row * 128;
+        // table[g][pos] = (cos, sin) of j = 2g and 2g + 1: consecutive rows read consecutive 16 bytes
+        const float4* tab = reinterpret_cast<const float4*>(args.rope_table) + pos;
+        float4 cs[kUnits / 2][4];                      // all table loads first: one L2 round trip
+#pragma unroll
+        for (int uu = 0; uu < kUnits / 2; ++uu)
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            cs[uu][i] = __ldg(tab + (size_t)((h * (kUnits / 2) + uu) * 4 + i) * (size_t)args.capacity);
+#pragma unroll
+        for (int uu = 0; uu < kUnits / 2; ++uu) {
+          const int u = h * (kUnits / 2) + uu;         // pairs (8u .. 8u+7, + D/2)
+          const uint32_t a_lo = q_row + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4);
+          const uint32_t a_hi = (D == 128)
+              ? q_row + (BM * 128) + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4)
+              : q_row + ((((uint32_t)(u + kUnits)) ^ ((uint32_t)row & 7u)) << 4);
+          uint32_t lo[4], hi[4];
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo[0]), "=r"(lo[1]), "=r"(lo[2]), "=r"(lo[3]) : "r"(a_lo));
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi[0]), "=r"(hi[1]), "=r"(hi[2]), "=r"(hi[3]) : "r"(a_hi));
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float4 c = cs[uu][i];                // (cos, sin) of two consecutive j
+            const __nv_bfloat162 l2 = *reinterpret_cast<__nv_bfloat162*>(&lo[i]);
+            const __nv_bfloat162 h2 = *reinterpret_cast<__nv_bfloat162*>(&hi[i]);
+            const float2 a = __bfloat1622float2(l2), b = __bfloat1622float2(h2);
+            lo[i] = pack_bf16(__fmaf_rn(a.x, c.x, -__fmul_rn(b.x, c.y)), __fmaf_rn(a.y, c.z, -__fmul_rn(b.y, c.w)));
+            hi[i] = pack_bf16(__fmaf_rn(b.x, c.x, __fmul_rn(a.x, c.y)), __fmaf_rn(b.y, c.z, __fmul_rn(a.y, c.w)));
+          }
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_lo), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_hi), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
+      }
+      mbar_arrive(bar_q_rot + 8 * t);
+      return true;
+    };
     while (true) {
       // in independent mode slot t has its own ring, and an item describes one tile (its slot-0 fields)
       const uint32_t ring = (kIndep ? (uint32_t)t * kRing : 0u) + it_n % kRing;
@@ -772,41 +815,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         key_hi = i_row;
       }
-      if (args.rope_table) {
-        // Fused path: rotate this row's part of the Q tile in shared memory (restart position =
-        // row - start of its prompt), same fp32 arithmetic and rounding as the stand-alone kernel.
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * t, it_n & 1u, wctx, kWaitQFull));
+      PROF_LAP(8);
+      // Fused path: Q arrives raw and is rotated in shared memory. In independent mode the rotation
+      // of item i+1 was already done before the epilogue of item i (see below), except for the
+      // first item.
+      if (args.rope_table && (!kIndep || it_n == 0)) {
+        ok = rotate_q(used ? key_hi - key_lo : -1, it_n & 1u);
         if (!ok) break;
-        const int pos = key_hi - key_lo;               // < 0 for padding rows (key_hi = 0, key_lo = 1)
-        if (used && pos > 0) {
-          constexpr int kUnits = D / 16;               // 16-byte units per half of a row
-          const uint32_t q_row = s_q + (uint32_t)t * Cfg::kQBytes + (uint32_t)row * 128;
-          const float4* tab = reinterpret_cast<const float4*>(args.rope_table + (size_t)pos * (D / 2));
-#pragma unroll
-          for (int uu = 0; uu < kUnits / 2; ++uu) {
-            const int u = h * (kUnits / 2) + uu;       // pairs (8u .. 8u+7, + D/2)
-            const uint32_t a_lo = q_row + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4);
-            const uint32_t a_hi = (D == 128)
-                ? q_row + (BM * 128) + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4)
-                : q_row + ((((uint32_t)(u + kUnits)) ^ ((uint32_t)row & 7u)) << 4);
-            uint32_t lo[4], hi[4];
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo[0]), "=r"(lo[1]), "=r"(lo[2]), "=r"(lo[3]) : "r"(a_lo));
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi[0]), "=r"(hi[1]), "=r"(hi[2]), "=r"(hi[3]) : "r"(a_hi));
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float4 cs = __ldg(tab + u * 4 + i);   // (cos, sin) of two consecutive j
-              const __nv_bfloat162 l2 = *reinterpret_cast<__nv_bfloat162*>(&lo[i]);
-              const __nv_bfloat162 h2 = *reinterpret_cast<__nv_bfloat162*>(&hi[i]);
-              const float2 a = __bfloat1622float2(l2), b = __bfloat1622float2(h2);
-              lo[i] = pack_bf16(__fmaf_rn(a.x, cs.x, -__fmul_rn(b.x, cs.y)), __fmaf_rn(a.y, cs.z, -__fmul_rn(b.y, cs.w)));
-              hi[i] = pack_bf16(__fmaf_rn(b.x, cs.x, __fmul_rn(a.x, cs.y)), __fmaf_rn(b.y, cs.z, __fmul_rn(a.y, cs.w)));
-            }
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_lo), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_hi), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-          }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
-        }
-        mbar_arrive(bar_q_rot + 8 * t);
+        PROF_LAP(11);
       }
       float m_run = -INFINITY;      // running maximum of the whole row, in scaled log2 units
       float l_run = 0.f;            // this thread's share of the running sum of exp2(s * c - m_run)
@@ -938,6 +954,31 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       if (!ok) break;
 
+      if (kIndep && args.rope_table) {
+        // Independent mode, fused path: while this item's last P V product is still running, get the
+        // next item's Q ready, so that its first S tile is computed under this item's epilogue.
+        const uint32_t nring = (uint32_t)t * kRing + (it_n + 1) % kRing;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * nring, ((it_n + 1) / kRing) & 1u, wctx, kWaitItemFull));
+        if (!ok) break;
+        const volatile int* ne = s_ring + nring * kRingInts;   // peeked, not consumed here
+        if (ne[0] >= 0) {
+          const int n_row = ne[4] + row;
+          int n_pos = -1;
+          if (n_row < ne[12]) {
+            int n_lo = ne[14];
+            if (!(ne[18] & 1)) {
+              for (int sg = ne[16] + 1; sg < ne[13]; ++sg) {
+                const int st = __ldg(tb + args.off_seg_start + sg);
+                if (st > n_row) break;
+                n_lo = st;
+              }
+            }
+            n_pos = n_row - n_lo;
+          }
+          ok = rotate_q(n_pos, (it_n + 1) & 1u);
+          if (!ok) break;
+        }
+      }
       // epilogue: O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store
       PROF_LAP(5);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full + 8 * t, it_n & 1u, wctx, kWaitOFull));

@@ -55,9 +55,11 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
 int note_cuda_error(int cuda_error, const char* what);
 
 // Kernel launchers (device pointers, stream = cudaStream_t as void*). Return a PP_* status.
+// Rotates the n_q_heads heads of q into q_out (may be the same buffer) and the n_kv_heads heads of k
+// in place; pass n_q_heads or n_kv_heads = 0 in `p` to rotate only the other tensor.
 int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L,
-                void* q, void* k, void* stream);
-// rope_table: device [capacity][D/2] (cos, sin) pairs, or null. When given, q holds the raw
+                const void* q, void* q_out, void* k, void* stream);
+// rope_table: device [D/4][capacity][2] (cos, sin) pairs, or null. When given, q holds the raw
 // queries and the kernel rotates each Q tile in shared memory before use.
 int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayout& L,
                      const void* q, const void* k, const void* v, void* o, const void* rope_table,

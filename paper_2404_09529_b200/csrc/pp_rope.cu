@@ -43,7 +43,7 @@ __device__ __forceinline__ void rotate8(uint4& lo, uint4& hi, const float* cs, c
 
 template <int D>
 __global__ void __launch_bounds__(kRopeThreads)
-rope_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k,
+rope_kernel(const __nv_bfloat16* q, __nv_bfloat16* q_out, __nv_bfloat16* __restrict__ k,
             const int32_t* __restrict__ table, int32_t off_bin_seg_ptr, int32_t off_bin_used,
             int32_t off_seg_start, int32_t n_bins, int32_t capacity, int32_t n_q_heads,
             int32_t n_kv_heads, const __grid_constant__ RopeFreq freq) {
@@ -99,24 +99,27 @@ rope_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k,
   for (int u = tid; u < kRopeRows * units_per_row; u += kRopeThreads) {
     const int r = u / units_per_row;
     const int w = u - r * units_per_row;
-    if (s_pos[r] <= 0) continue;                    // padding row, or position 0 (identity)
+    const bool in_place = (q_out == q);
+    // padding rows are skipped; position 0 is the identity (copied only when Q goes elsewhere)
+    if (s_pos[r] < 0 || (s_pos[r] == 0 && (in_place || w >= n_q_heads * kUnitsPerHead))) continue;
     const int head = w / kUnitsPerHead;
     const int c = w - head * kUnitsPerHead;
     const int64_t row = row0 + r;
-    __nv_bfloat16* base = head < n_q_heads
-        ? q + (row * n_q_heads + head) * D
-        : k + (row * n_kv_heads + (head - n_q_heads)) * D;
-    uint4* p_lo = reinterpret_cast<uint4*>(base + c * 8);
-    uint4* p_hi = reinterpret_cast<uint4*>(base + kHalf + c * 8);
-    uint4 lo = *p_lo, hi = *p_hi;
-    rotate8(lo, hi, &s_cos[r][c * 8], &s_sin[r][c * 8]);
-    *p_lo = lo;
-    *p_hi = hi;
+    const bool is_q = head < n_q_heads;
+    const int64_t off = is_q ? (row * n_q_heads + head) * D : (row * n_kv_heads + (head - n_q_heads)) * D;
+    const __nv_bfloat16* src = is_q ? q + off : k + off;
+    __nv_bfloat16* dst = is_q ? q_out + off : k + off;
+    uint4 lo = *reinterpret_cast<const uint4*>(src + c * 8);
+    uint4 hi = *reinterpret_cast<const uint4*>(src + kHalf + c * 8);
+    if (s_pos[r] > 0) rotate8(lo, hi, &s_cos[r][c * 8], &s_sin[r][c * 8]);
+    *reinterpret_cast<uint4*>(dst + c * 8) = lo;
+    *reinterpret_cast<uint4*>(dst + kHalf + c * 8) = hi;
   }
 }
 
-// cos/sin of position * theta_j for every position of a bin: table[pos][j] = (cos, sin). Read by
-// the attention kernel, which rotates Q on the fly in the fused path.
+// cos/sin of position * theta_j for every position of a bin, laid out [j / 2][pos][j % 2] as
+// (cos, sin) pairs, so that threads working on consecutive rows (positions) read consecutive
+// 16-byte pieces. Read by the fused kernels.
 __global__ void __launch_bounds__(256)
 rope_table_kernel(float2* __restrict__ table, int32_t capacity, int32_t half,
                   const __grid_constant__ RopeFreq freq) {
@@ -131,7 +134,7 @@ rope_table_kernel(float2* __restrict__ table, int32_t capacity, int32_t half,
     red = fma(-n, 2.4492935982947064e-16, red);
     sincosf((float)red, &sn, &cs);
   }
-  table[idx] = make_float2(cs, sn);
+  table[((size_t)(j >> 1) * capacity + pos) * 2 + (j & 1)] = make_float2(cs, sn);
 }
 
 // Fused K rotation + UNPACK (Algorithm 1 lines 7-8 in one pass over K and V): every real packed
@@ -185,43 +188,70 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
   }
   __syncthreads();
 
-  const int units_k = n_kv_heads * kPairUnits;
+  // V rows first: plain 16-byte copies, four in flight per thread
   const int units_v = n_kv_heads * kVecs;
-  const int units_per_row = units_k + units_v;
-  for (int u = tid; u < kRopeRows * units_per_row; u += kRopeThreads) {
-    const int r = u / units_per_row;
-    int w = u - r * units_per_row;
-    const int32_t pos = s_pos[r];
-    if (pos < 0) continue;                          // padding row
-    const int64_t row = row0 + r;
-    const int64_t dst = s_dst[r];
-    if (w < units_k) {
-      const int head = w / kPairUnits, c = w - head * kPairUnits;
-      __nv_bfloat16* base = k + (row * n_kv_heads + head) * D;
-      uint4 lo = *reinterpret_cast<const uint4*>(base + c * 8);
-      uint4 hi = *reinterpret_cast<const uint4*>(base + kHalf + c * 8);
+  for (int u0 = tid; u0 < kRopeRows * units_v; u0 += 4 * kRopeThreads) {
+    uint4 val[4];
+    int64_t dsts[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int u = u0 + i * kRopeThreads;
+      dsts[i] = -1;
+      if (u < kRopeRows * units_v) {
+        const int r = u / units_v, w = u - r * units_v;
+        if (s_dst[r] >= 0) {
+          const int head = w / kVecs, c = w - head * kVecs;
+          val[i] = __ldg(reinterpret_cast<const uint4*>(v + ((row0 + r) * n_kv_heads + head) * D + c * 8));
+          dsts[i] = s_dst[r] + head * s_head_stride[r] + c * 8;
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (dsts[i] >= 0) *reinterpret_cast<uint4*>(v_cache + dsts[i]) = val[i];
+  }
+  // K rows: rotate, write back to the packed tensor and into the cache; two pairs in flight
+  const int units_k = n_kv_heads * kPairUnits;
+  for (int u0 = tid; u0 < kRopeRows * units_k; u0 += 2 * kRopeThreads) {
+    uint4 lo[2], hi[2];
+    int rr[2], hh[2], cc[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int u = u0 + i * kRopeThreads;
+      rr[i] = -1;
+      if (u < kRopeRows * units_k) {
+        const int r = u / units_k, w = u - r * units_k;
+        if (s_pos[r] >= 0) {
+          rr[i] = r; hh[i] = w / kPairUnits; cc[i] = w - hh[i] * kPairUnits;
+          const __nv_bfloat16* base = k + ((row0 + r) * n_kv_heads + hh[i]) * D;
+          lo[i] = *reinterpret_cast<const uint4*>(base + cc[i] * 8);
+          hi[i] = *reinterpret_cast<const uint4*>(base + kHalf + cc[i] * 8);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      if (rr[i] < 0) continue;
+      const int r = rr[i], head = hh[i], c = cc[i];
+      const int32_t pos = s_pos[r];
+      __nv_bfloat16* base = k + ((row0 + r) * n_kv_heads + head) * D;
       if (pos > 0) {
         float cs[8], sn[8];
-        const float4* tab = reinterpret_cast<const float4*>(rope_table + (size_t)pos * kHalf + c * 8);
+        const float4* tab = reinterpret_cast<const float4*>(rope_table) + pos;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float4 t4 = __ldg(tab + i);
-          cs[2 * i] = t4.x; sn[2 * i] = t4.y; cs[2 * i + 1] = t4.z; sn[2 * i + 1] = t4.w;
+        for (int q = 0; q < 4; ++q) {
+          const float4 t4 = __ldg(tab + (size_t)(c * 4 + q) * (size_t)capacity);
+          cs[2 * q] = t4.x; sn[2 * q] = t4.y; cs[2 * q + 1] = t4.z; sn[2 * q + 1] = t4.w;
         }
-        rotate8(lo, hi, cs, sn);
-        *reinterpret_cast<uint4*>(base + c * 8) = lo;
-        *reinterpret_cast<uint4*>(base + kHalf + c * 8) = hi;
+        rotate8(lo[i], hi[i], cs, sn);
+        *reinterpret_cast<uint4*>(base + c * 8) = lo[i];
+        *reinterpret_cast<uint4*>(base + kHalf + c * 8) = hi[i];
       }
-      if (dst >= 0) {
-        __nv_bfloat16* cd = k_cache + dst + head * s_head_stride[r];
-        *reinterpret_cast<uint4*>(cd + c * 8) = lo;
-        *reinterpret_cast<uint4*>(cd + kHalf + c * 8) = hi;
+      if (s_dst[r] >= 0) {
+        __nv_bfloat16* cd = k_cache + s_dst[r] + head * s_head_stride[r];
+        *reinterpret_cast<uint4*>(cd + c * 8) = lo[i];
+        *reinterpret_cast<uint4*>(cd + kHalf + c * 8) = hi[i];
       }
-    } else if (dst >= 0) {
-      w -= units_k;
-      const int head = w / kVecs, c = w - head * kVecs;
-      const uint4 val = __ldg(reinterpret_cast<const uint4*>(v + (row * n_kv_heads + head) * D + c * 8));
-      *reinterpret_cast<uint4*>(v_cache + dst + head * s_head_stride[r] + c * 8) = val;
     }
   }
 }
@@ -266,19 +296,19 @@ int launch_rope_unpack(const pp_attn_params& p, const int32_t* d_table, const Ta
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "rope+unpack kernel launch");
 }
 
-int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L, void* q,
-                void* k, void* stream) {
+int launch_rope(const pp_attn_params& p, const int32_t* d_table, const TableLayout& L, const void* q,
+                void* q_out, void* k, void* stream) {
   const RopeFreq freq = make_freq(p);
   const int64_t n_rows = (int64_t)p.n_bins * p.capacity;
   const unsigned grid = (unsigned)((n_rows + kRopeRows - 1) / kRopeRows);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p.head_dim == 128) {
     rope_kernel<128><<<grid, kRopeThreads, 0, s>>>(
-        (__nv_bfloat16*)q, (__nv_bfloat16*)k, d_table, L.bin_seg_ptr, L.bin_used, L.seg_start,
+        (const __nv_bfloat16*)q, (__nv_bfloat16*)q_out, (__nv_bfloat16*)k, d_table, L.bin_seg_ptr, L.bin_used, L.seg_start,
         p.n_bins, p.capacity, p.n_q_heads, p.n_kv_heads, freq);
   } else {
     rope_kernel<64><<<grid, kRopeThreads, 0, s>>>(
-        (__nv_bfloat16*)q, (__nv_bfloat16*)k, d_table, L.bin_seg_ptr, L.bin_used, L.seg_start,
+        (const __nv_bfloat16*)q, (__nv_bfloat16*)q_out, (__nv_bfloat16*)k, d_table, L.bin_seg_ptr, L.bin_used, L.seg_start,
         p.n_bins, p.capacity, p.n_q_heads, p.n_kv_heads, freq);
   }
   const cudaError_t e = cudaGetLastError();
