@@ -4,17 +4,26 @@
 // row carries the key range [start row of its prompt, its own row], and the host work list
 // restricts each query tile to the key tiles that can intersect such a range.
 //
-// Persistent kernel, one CTA per SM, 640 threads. Each CTA draws work items from a global counter
-// (items are listed KV-head-major, longest first). A work item has two 128-row query-tile slots
-// that share one stream of 128-row key/value tiles: two query heads of one KV head over the same
-// rows (even GQA group), or two consecutive row tiles of one head.
+// Persistent kernel, one CTA per SM, 640 threads, two 128-row query-tile slots per CTA. CTAs draw
+// work from a global counter (items are listed KV-head-major, longest first). Two modes, chosen on
+// the host from the mean number of key tiles per query tile:
+//
+// Shared-stream mode (long items). A work item has two slots that share one stream of 128-row
+// key/value tiles: two query heads of one KV head over the same rows (even GQA group), or two
+// consecutive row tiles of one head.
 //   warp 0       draws and decodes items, TMA-loads the K / V tile rings
 //   warp 1       issues tcgen05.mma: S_t = Q_t K^T into TMEM, O_t += P_t V with P_t read from TMEM;
 //                the two slots alternate so that one slot's MMAs run while the other's softmax works
 //   warps 2-3    TMA-load Q of slot 0 / slot 1
-//   warps 4-11   softmax of slot 0: two threads per query row (TMEM lane = row), one per 64-key half
+// Independent mode (short items). Every slot draws its own items (one query tile each) and walks
+// their 64-row key tiles on its own; S_t has two 64-column buffers so that the scores of tile k+1
+// and the product P(k) V(k) are computed while the softmax threads work.
+//   warps 0-1    issue the tcgen05.mma of slot 0 / slot 1
+//   warps 2-3    draw items and TMA-load Q, K, V of slot 0 / slot 1 (two K and two V stages each)
+// Both modes:
+//   warps 4-11   softmax of slot 0: two threads per query row (TMEM lane = row), one per half tile
 //   warps 12-19  softmax of slot 1
-// Softmax: tcgen05.ld the thread's 64 scores, mask to the row's key range, row maximum exchanged
+// Softmax: tcgen05.ld the thread's scores, mask to the row's key range, row maximum exchanged
 // between the two halves through shared memory, lazy running maximum (O is rescaled only when
 // the maximum grows by more than 2^8), exp2, P written as bf16 over the S columns; at the end of
 // an item O / l goes through a swizzled staging buffer and a TMA store.
@@ -34,25 +43,26 @@ namespace pp {
 namespace {
 
 constexpr int BM = kTileM;
-constexpr int BN = kTileN;
 constexpr int kAttnThreads = 640;
 constexpr int kSoftmaxThreads = 256;       // per slot: two threads per query row
 constexpr uint32_t kTmemCols = 512;
 constexpr int kRegsSoftmax = 104;          // setmaxnreg budgets: 640 threads start with 96 registers each;
 constexpr int kRegsOther = 64;              // warps 0-3 give back 32 each, the 512 softmax threads take 8 each
-constexpr uint32_t kRing = 4;               // decoded work items in flight between the fetching thread and its readers
+constexpr uint32_t kRing = 3;               // decoded work items in flight between the fetching thread and its readers
 constexpr int kRingInts = 20;              // ints per ring entry
 
-template <int D> struct AttnCfg {
-  static constexpr int kKStages = (D == 128) ? 2 : 4;
-  static constexpr int kVStages = (D == 128) ? 2 : 4;
+// BN: key rows per tile. 128 in shared-stream mode; 64 in independent mode, where every slot owns
+// two K and two V stages and two S buffers (see the kernel).
+template <int D, int BN> struct AttnCfg {
+  static constexpr int kKStages = (D == 128 && BN == 128) ? 2 : 4;
+  static constexpr int kVStages = (D == 128 && BN == 128) ? 2 : 4;
   static constexpr int kChunks = D / 64;                     // 128-byte swizzle spans per row
   static constexpr int kQBytes = BM * D * 2;                 // per slot
   static constexpr int kKVBytes = BN * D * 2;
-  static constexpr int kStageOBytes = BM * 128;              // per slot: one 64-column box of O
-  // barriers + work ring (768) and the row-maximum exchange buffer [slot][half][row] (2048), placed
+  // barriers + work ring (1024) and the row-maximum exchange buffer [slot][half][row] (2048), placed
   // in front of the 1024-byte-aligned tiles; at D = 128 the total is exactly the 227 KB limit
   static constexpr int kMiscBytes = 3072;
+  static constexpr int kStageOBytes = BM * 128;              // per slot: one 64-column box of O
   static constexpr int kTileBytes = 2 * kQBytes + (kKStages + kVStages) * kKVBytes + 2 * kStageOBytes;
   static constexpr int kSmemBytes = kMiscBytes + kTileBytes;
   static constexpr uint32_t kTmemS = 0;                      // S_t at 128 * t
@@ -338,14 +348,15 @@ enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWai
 
 // kIndep = false: the two slots of a CTA work on one item and share its K/V stream (long
 //   sequences, GQA head pairs). kIndep = true: every slot draws its own single-tile items and loads
-//   its own K/V tiles, so neither slot ever waits for the other (short prompts, where pairing two
-//   row tiles of different length would leave one slot idle for a tile per item).
+//   its own K/V tiles (64 rows each), so neither slot ever waits for the other (short prompts, where
+//   pairing two row tiles of different length would leave one slot idle for a tile per item).
 template <int D, bool kIndep>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                  const AttnArgs args) {
-  using Cfg = AttnCfg<D>;
+  constexpr int BN = kIndep ? kTileNShort : kTileN;
+  using Cfg = AttnCfg<D, BN>;
   constexpr int NK = Cfg::kKStages, NV = Cfg::kVStages, kChunks = Cfg::kChunks;
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -368,20 +379,20 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const uint32_t bar_item_empty = s_misc + 64;   // [2 rings][kRing]
   const uint32_t bar_q_full = s_misc + 128;      // [2]
   const uint32_t bar_q_empty = s_misc + 144;     // [2]
-  const uint32_t bar_s_full = s_misc + 160;      // [2]
-  const uint32_t bar_p_full = s_misc + 176;      // [2]
-  const uint32_t bar_o_full = s_misc + 192;      // [2]
-  const uint32_t bar_o_empty = s_misc + 208;     // [2]
-  const uint32_t bar_k_full = s_misc + 224;      // [4]
-  const uint32_t bar_k_empty = s_misc + 256;     // [4]
-  const uint32_t bar_v_full = s_misc + 288;      // [4]
-  const uint32_t bar_v_empty = s_misc + 320;     // [4]
-  volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 352);   // [2 rings][kRing][kRingInts]
-  const uint32_t bar_q_rot = s_misc + 1000;      // [2] Q_t has been rotated in place (fused path)
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 992);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 996);
+  const uint32_t bar_s_full = s_misc + 160;      // [2 slots][2 S buffers]; shared mode uses [t][0]
+  const uint32_t bar_p_full = s_misc + 192;      // [2 slots][2 S buffers]
+  const uint32_t bar_o_full = s_misc + 224;      // [2]
+  const uint32_t bar_o_empty = s_misc + 240;     // [2]
+  const uint32_t bar_k_full = s_misc + 256;      // [4]; independent mode: [2 slots][2 stages]
+  const uint32_t bar_k_empty = s_misc + 288;     // [4]
+  const uint32_t bar_v_full = s_misc + 320;      // [4]
+  const uint32_t bar_v_empty = s_misc + 352;     // [4]
+  const uint32_t bar_q_rot = s_misc + 384;       // [2] Q_t has been rotated in place (fused path)
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 400);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 404);
+  volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 416);   // [2 rings][kRing][kRingInts]
   volatile float* s_xchg = reinterpret_cast<volatile float*>(misc + 1024);   // [2 slots][2 halves][128 rows]
-  static_assert(352 + 2 * kRing * kRingInts * 4 <= 992, "ring does not fit");
+  static_assert(416 + 2 * kRing * kRingInts * 4 <= 1024, "ring does not fit");
   static_assert(NK <= 4 && NV <= 4, "barrier slots");
 
   const int warp = threadIdx.x >> 5;
@@ -399,8 +410,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_init(bar_q_full + 8 * i, 1);
       mbar_init(bar_q_empty + 8 * i, 1);
       mbar_init(bar_q_rot + 8 * i, kSoftmaxThreads);
-      mbar_init(bar_s_full + 8 * i, 1);
-      mbar_init(bar_p_full + 8 * i, kSoftmaxThreads);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(bar_s_full + 8 * (2 * i + b), 1);
+        mbar_init(bar_p_full + 8 * (2 * i + b), kSoftmaxThreads);
+      }
       mbar_init(bar_o_full + 8 * i, 1);
       mbar_init(bar_o_empty + 8 * i, kSoftmaxThreads / 2);   // the half-0 threads run the epilogue
     }
@@ -452,108 +465,107 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           bool ok = true;
           for (int j = 0; ok && j < wk.n; ++j, ++kc) {
             const int kv0 = wk.kv_row0 + j * BN;
-            ok = mbar_wait(bar_k_empty + 8 * t, (kc & 1u) ^ 1u, wctx, kWaitKEmpty);
+            const uint32_t st = 2u * (uint32_t)t + (kc & 1u);          // the slot's stage for this tile
+            const uint32_t free_parity = ((kc >> 1) & 1u) ^ 1u;
+            ok = mbar_wait(bar_k_empty + 8 * st, free_parity, wctx, kWaitKEmpty);
             if (!ok) break;
-            mbar_expect_tx(bar_k_full + 8 * t, Cfg::kKVBytes);
+            mbar_expect_tx(bar_k_full + 8 * st, Cfg::kKVBytes);
             for (int c = 0; c < kChunks; ++c)
-              tma_load_4d(s_k + t * Cfg::kKVBytes + c * (BN * 128), &map_k, bar_k_full + 8 * t,
+              tma_load_4d(s_k + st * Cfg::kKVBytes + c * (BN * 128), &map_k, bar_k_full + 8 * st,
                           c * 64, wk.kv_head, kv0, wk.bin);
-            ok = mbar_wait(bar_v_empty + 8 * t, (kc & 1u) ^ 1u, wctx, kWaitVEmpty);
+            ok = mbar_wait(bar_v_empty + 8 * st, free_parity, wctx, kWaitVEmpty);
             if (!ok) break;
-            mbar_expect_tx(bar_v_full + 8 * t, Cfg::kKVBytes);
+            mbar_expect_tx(bar_v_full + 8 * st, Cfg::kKVBytes);
             for (int c = 0; c < kChunks; ++c)
-              tma_load_4d(s_v + t * Cfg::kKVBytes + c * (BN * 128), &map_v, bar_v_full + 8 * t,
+              tma_load_4d(s_v + st * Cfg::kKVBytes + c * (BN * 128), &map_v, bar_v_full + 8 * st,
                           c * 64, wk.kv_head, kv0, wk.bin);
           }
           if (!ok) break;
           ++it_n;
         }
-      } else if (warp == 1 && lane == 0) {
-        // -------------------------------------------------------------- MMA issuer, independent slots
-        // Each slot walks  item -> S(0) -> [P V(j), S(j+1)] ... -> end of item  on its own; the
-        // thread polls both and issues whichever next step is ready.
+      } else if (warp < 2 && lane == 0) {
+        // -------------------------------------------------------------- MMA issuer of slot t
+        // One issuing thread per slot (warps 0 and 1 sit on different schedulers), plain blocking
+        // waits. S_t has two 64-column buffers, tile k of the slot's stream uses buffer k & 1, and
+        // P(k) is written over S(k). The issue order  S(k+1), then P(k) V(k)  lets the tensor pipe
+        // compute the next scores while the softmax threads work on tile k, and P(k) V(k) while they
+        // work on tile k+1; the pipe runs one thread's MMAs in order, so S(k+2) cannot overwrite
+        // P(k) before P(k) V(k) has read it.
+        const int t = warp;
         constexpr uint32_t idesc_qk = instr_desc(BN, false);
         constexpr uint32_t idesc_pv = instr_desc(D, true);
-        const uint32_t q_lo0 = desc_lo(s_q, 0), k_lo0 = desc_lo(s_k, 0), v_lo0 = desc_lo(s_v, BN * 128);
-        const uint32_t bar_q_ready = args.rope_table ? bar_q_rot : bar_q_full;
-        enum { kNeedItem = 0, kNeedS, kNeedPV, kDone };
-        uint32_t itn0 = 0, kcn0 = 0, itn1 = 0, kcn1 = 0;   // items and key tiles consumed per slot
-        int st0 = kNeedItem, j0 = 0, n0 = 0, st1 = kNeedItem, j1 = 0, n1 = 0;
-#define PP_INDEP_STEP(T, ITN_, KCN_, ST_, J_, NT_)                                                      \
-  [&]() -> bool {                                                                                       \
-    if (ST_ == kNeedPV) {                                                                               \
-      /* the previous item's epilogue must have read O_T before it is overwritten */                    \
-      if (J_ == 0 && !mbar_try_wait(bar_o_empty + 8 * T, (ITN_ & 1u) ^ 1u)) return false;               \
-      if (!mbar_try_wait(bar_p_full + 8 * T, KCN_ & 1u)) return false;                                  \
-      if (!mbar_try_wait(bar_v_full + 8 * T, KCN_ & 1u)) return false;                                  \
-      tc_fence_after(); /* O_T (+)= P_T V_j */                                                          \
-      const uint32_t a = tmem_base + Cfg::kTmemS + 128u * T;                                            \
-      const uint32_t d = tmem_base + Cfg::kTmemO + (uint32_t)D * T;                                     \
-      const uint32_t b_lo = v_lo0 + (uint32_t)T * (Cfg::kKVBytes >> 4);                                 \
-      mma_ts(d, a, b_lo, idesc_pv, J_ == 0 ? 0u : 1u);                                                  \
-      _Pragma("unroll") for (int kk = 1; kk < BN / 16; ++kk)                                            \
-        mma_ts(d, a + kk * 8, b_lo + (uint32_t)kk * ((16 * 128) >> 4), idesc_pv, 1u);                   \
-      tc_commit(bar_v_empty + 8 * T);                                                                   \
-      ++KCN_;                                                                                           \
-      if (++J_ == NT_) {                                                                                \
-        tc_commit(bar_o_full + 8 * T);                                                                  \
-        ++ITN_;                                                                                         \
-        ST_ = kNeedItem;                                                                                \
-      } else {                                                                                          \
-        ST_ = kNeedS;                                                                                   \
-      }                                                                                                 \
-      return true;                                                                                      \
-    }                                                                                                   \
-    if (ST_ == kNeedS) {                                                                                \
-      if (J_ == 0 && !mbar_try_wait(bar_q_ready + 8 * T, ITN_ & 1u)) return false;                      \
-      if (!mbar_try_wait(bar_k_full + 8 * T, KCN_ & 1u)) return false;                                  \
-      tc_fence_after(); /* S_T = Q_T K_j^T */                                                           \
-      const uint32_t d = tmem_base + Cfg::kTmemS + 128u * T;                                            \
-      const uint32_t a_lo = q_lo0 + (uint32_t)T * (Cfg::kQBytes >> 4);                                  \
-      const uint32_t b_lo = k_lo0 + (uint32_t)T * (Cfg::kKVBytes >> 4);                                 \
-      _Pragma("unroll") for (int kk = 0; kk < D / 16; ++kk) {                                           \
-        constexpr uint32_t kChunkQ = (BM * 128) >> 4, kChunkK = (BN * 128) >> 4;                        \
-        mma_ss(d, a_lo + (uint32_t)(kk >> 2) * kChunkQ + (uint32_t)(kk & 3) * 2,                        \
-               b_lo + (uint32_t)(kk >> 2) * kChunkK + (uint32_t)(kk & 3) * 2, idesc_qk,                 \
-               kk > 0 ? 1u : 0u);                                                                       \
-      }                                                                                                 \
-      tc_commit(bar_k_empty + 8 * T);                                                                   \
-      tc_commit(bar_s_full + 8 * T);                                                                    \
-      if (J_ + 1 == NT_) tc_commit(bar_q_empty + 8 * T); /* last read of Q_T in this item */            \
-      ST_ = kNeedPV;                                                                                    \
-      return true;                                                                                      \
-    }                                                                                                   \
-    if (ST_ == kNeedItem) {                                                                             \
-      const uint32_t ring = ITN_ % kRing;                                                               \
-      if (!mbar_try_wait(bar_item_full + 8 * (T * kRing + ring), (ITN_ / kRing) & 1u)) return false;    \
-      const volatile int* e = s_ring + (T * (int)kRing + (int)ring) * kRingInts;                        \
-      const int w = e[0];                                                                               \
-      NT_ = e[3];                                                                                       \
-      mbar_arrive(bar_item_empty + 8 * (T * kRing + ring));                                             \
-      if (w < 0) { ST_ = kDone; return true; }                                                          \
-      J_ = 0;                                                                                           \
-      ST_ = kNeedS;                                                                                     \
-      return true;                                                                                      \
-    }                                                                                                   \
-    return false;                                                                                       \
-  }()
-        unsigned long long idle_since = 0;
-        uint32_t idle_spins = 0;
-        while (st0 != kDone || st1 != kDone) {
-          const bool a0 = PP_INDEP_STEP(0, itn0, kcn0, st0, j0, n0);
-          const bool a1 = PP_INDEP_STEP(1, itn1, kcn1, st1, j1, n1);
-          if (a0 || a1) { idle_spins = 0; continue; }
-          if (idle_spins++ == 0) idle_since = global_ns();
-          if ((idle_spins & 255u) == 0) {           // bounded: give up like every other wait
-            if (*s_abort) break;
-            if (global_ns() - idle_since > wctx.limit_ns) {
-              *s_abort = 1;
-              if (wctx.status) atomicCAS(wctx.status, 0, (int)kWaitP);
-              break;
-            }
+        const uint32_t a_lo = desc_lo(s_q, 0) + (uint32_t)t * (Cfg::kQBytes >> 4);
+        const uint32_t k_lo = desc_lo(s_k, 0) + 2u * (uint32_t)t * (Cfg::kKVBytes >> 4);
+        const uint32_t v_lo = desc_lo(s_v, BN * 128) + 2u * (uint32_t)t * (Cfg::kKVBytes >> 4);
+        const uint32_t tm_s = tmem_base + Cfg::kTmemS + 128u * (uint32_t)t;
+        const uint32_t tm_o = tmem_base + Cfg::kTmemO + (uint32_t)D * (uint32_t)t;
+        const uint32_t bar_q_ready = (args.rope_table ? bar_q_rot : bar_q_full) + 8 * t;
+        const uint32_t b_item_full = bar_item_full + 8 * (uint32_t)t * kRing;
+        const uint32_t b_item_empty = bar_item_empty + 8 * (uint32_t)t * kRing;
+        const uint32_t b_k_full = bar_k_full + 16 * t, b_k_empty = bar_k_empty + 16 * t;   // [stage]
+        const uint32_t b_v_full = bar_v_full + 16 * t, b_v_empty = bar_v_empty + 16 * t;
+        const uint32_t b_s_full = bar_s_full + 16 * t, b_p_full = bar_p_full + 16 * t;     // [buffer]
+        const uint32_t b_o_full = bar_o_full + 8 * t, b_o_empty = bar_o_empty + 8 * t;
+        const uint32_t b_q_empty = bar_q_empty + 8 * t;
+        uint32_t it_n = 0, kc = 0;       // items and key tiles consumed
+        bool ok = true;
+        PROF_DECL(8);
+        // S(kq) = Q_t K(kq)^T into buffer kq & 1
+        auto issue_qk = [&](const uint32_t kq, const bool last_of_item) -> bool {
+          const uint32_t b = kq & 1u;
+          if (!mbar_wait(b_k_full + 8 * b, (kq >> 1) & 1u, wctx, kWaitKFull)) return false;
+          PROF_LAP(2);
+          tc_fence_after();
+          const uint32_t d = tm_s + 64u * b;
+          const uint32_t kb = k_lo + b * (Cfg::kKVBytes >> 4);
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            constexpr uint32_t kChunkQ = (BM * 128) >> 4, kChunkK = (BN * 128) >> 4;
+            mma_ss(d, a_lo + (uint32_t)(kk >> 2) * kChunkQ + (uint32_t)(kk & 3) * 2,
+                   kb + (uint32_t)(kk >> 2) * kChunkK + (uint32_t)(kk & 3) * 2, idesc_qk, kk > 0 ? 1u : 0u);
           }
+          tc_commit(b_k_empty + 8 * b);
+          tc_commit(b_s_full + 8 * b);
+          if (last_of_item) tc_commit(b_q_empty);     // last read of Q_t in this item
+          PROF_LAP(3);
+          return true;
+        };
+        while (ok) {
+          const uint32_t ring = it_n % kRing;
+          if (!mbar_wait(b_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull)) break;
+          const volatile int* e = s_ring + (t * (int)kRing + (int)ring) * kRingInts;
+          const int w = e[0], n = e[3];
+          mbar_arrive(b_item_empty + 8 * ring);
+          if (w < 0) break;
+          PROF_LAP(0);
+          if (!(ok = mbar_wait(bar_q_ready, it_n & 1u, wctx, kWaitQFull))) break;
+          PROF_LAP(1);
+          if (!(ok = issue_qk(kc, n == 1))) break;
+          for (int j = 0; j < n; ++j, ++kc) {
+            if (j + 1 < n && !(ok = issue_qk(kc + 1, j + 2 == n))) break;
+            // the previous item's epilogue must have read O_t before it is overwritten
+            if (j == 0 && !(ok = mbar_wait(b_o_empty, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
+            PROF_LAP(4);
+            const uint32_t b = kc & 1u, parity = (kc >> 1) & 1u;
+            if (!(ok = mbar_wait(b_p_full + 8 * b, parity, wctx, kWaitP))) break;
+            PROF_LAP(5);
+            if (!(ok = mbar_wait(b_v_full + 8 * b, parity, wctx, kWaitVFull))) break;
+            PROF_LAP(6);
+            tc_fence_after();            // O_t (+)= P(k) V(k)
+            const uint32_t a = tm_s + 64u * b;
+            const uint32_t vb = v_lo + b * (Cfg::kKVBytes >> 4);
+            mma_ts(tm_o, a, vb, idesc_pv, j == 0 ? 0u : 1u);
+#pragma unroll
+            for (int kk = 1; kk < BN / 16; ++kk)
+              mma_ts(tm_o, a + kk * 8, vb + (uint32_t)kk * ((16 * 128) >> 4), idesc_pv, 1u);
+            tc_commit(b_v_empty + 8 * b);
+            PROF_LAP(7);
+          }
+          if (!ok) break;
+          tc_commit(b_o_full);
+          ++it_n;
         }
-#undef PP_INDEP_STEP
+        if (t == 0) PROF_STORE(0, 8);
       }
     } else {
     if (warp == 0 && lane == 0) {
@@ -648,7 +660,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                  b_lo + (uint32_t)(kk >> 2) * kChunkK + (uint32_t)(kk & 3) * 2, idesc_qk, kk > 0 ? 1u : 0u);
         }
         if (t == 1 || !(j >= jb1 && j < je1)) tc_commit(bar_k_empty + 8 * s);
-        tc_commit(bar_s_full + 8 * t);
+        tc_commit(bar_s_full + 16 * t);
         PROF_LAP(3);
         return true;
       };
@@ -660,7 +672,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // the previous item's epilogue must have read O_t before it is overwritten
           if (first && !mbar_wait(bar_o_empty + 8 * t, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty)) return false;
           PROF_LAP(4);
-          if (!mbar_wait(bar_p_full + 8 * t, tcount & 1u, wctx, kWaitP)) return false;
+          if (!mbar_wait(bar_p_full + 16 * t, tcount & 1u, wctx, kWaitP)) return false;
           PROF_LAP(5);
           const uint32_t vc = vc0 + (uint32_t)j, s = vc % NV;
           if (!mbar_wait(bar_v_full + 8 * s, (vc / NV) & 1u, wctx, kWaitVFull)) return false;
@@ -828,45 +840,50 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       float l_run = 0.f;            // this thread's share of the running sum of exp2(s * c - m_run)
 
       for (int j = jb_t; j < je_t; ++j) {
-        const int kv0 = item_kv_row0 + j * BN + 64 * h;      // first key of this thread's half
+        constexpr int EPT = BN / 2;                          // scores per thread and tile
+        constexpr int NCH = EPT / 32;                        // 32-column TMEM round trips
+        const int kv0 = item_kv_row0 + j * BN + EPT * h;     // first key of this thread's half
         const int c_lo = max(key_lo - kv0, 0);
-        const int c_hi = min(key_hi - kv0, 63);              // visible columns [c_lo, c_hi] of the half
-        const bool full = (c_lo == 0) && (c_hi == 63);
+        const int c_hi = min(key_hi - kv0, EPT - 1);         // visible columns [c_lo, c_hi] of the half
+        const bool full = (c_lo == 0) && (c_hi == EPT - 1);
         const bool warp_full = __all_sync(0xffffffffu, full);
-        const bool need0 = __any_sync(0xffffffffu, c_lo <= min(c_hi, 31));
-        const bool need1 = __any_sync(0xffffffffu, max(c_lo, 32) <= c_hi);
+        bool need[NCH];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch)
+          need[ch] = __any_sync(0xffffffffu, max(c_lo, 32 * ch) <= min(c_hi, 32 * ch + 31));
+        // independent mode: tile k of the slot's stream lives in S buffer k & 1
+        const uint32_t sbuf = kIndep ? (tcount & 1u) : 0u;
+        const uint32_t tparity = kIndep ? ((tcount >> 1) & 1u) : (tcount & 1u);
+        const uint32_t tmem_sb = tmem_s + 64u * sbuf;
         PROF_LAP(5);
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * t, tcount & 1u, wctx, kWaitS));
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * (2 * t + sbuf), tparity, wctx, kWaitS));
         if (!ok) break;                                      // warp-uniform
         tc_fence_after();
         PROF_LAP(1);
 
-        // this thread's 64 scores, one TMEM round trip
-        uint32_t v[64];
-        if (need0) {
-          tmem_ld32(tmem_s + 64 * h, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-        } else {
+        // this thread's scores
+        uint32_t v[EPT];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0xff800000u;                    // -inf
-        }
-        if (need1) {
-          tmem_ld32(tmem_s + 64 * h + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-        } else {
+        for (int ch = 0; ch < NCH; ++ch) {
+          if (need[ch]) {
+            tmem_ld32(tmem_sb + EPT * h + 32 * ch, *reinterpret_cast<uint32_t(*)[32]>(&v[32 * ch]));
+          } else {
 #pragma unroll
-          for (int i = 32; i < 64; ++i) v[i] = 0xff800000u;
+            for (int i = 0; i < 32; ++i) v[32 * ch + i] = 0xff800000u;        // -inf
+          }
         }
         tc_wait_ld();
         PROF_LAP(2);
         if (!warp_full) {
           // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
           // one of the two bounds (the causal diagonal, or the first tile of a prompt)
-          if (__any_sync(0xffffffffu, c_hi < 63)) {
+          if (__any_sync(0xffffffffu, c_hi < EPT - 1)) {
 #pragma unroll
-            for (int i = 0; i < 64; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
+            for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
           }
           if (__any_sync(0xffffffffu, c_lo > 0)) {
 #pragma unroll
-            for (int i = 0; i < 64; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
+            for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
           }
         }
         float mx;
@@ -876,15 +893,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           float m2 = fmax3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
           float m3 = fmax3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
 #pragma unroll
-          for (int i = 12; i + 7 < 64; i += 8) {
+          for (int i = 12; i + 7 < EPT; i += 8) {
             m0 = fmax3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
             m1 = fmax3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
             m2 = fmax3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
             m3 = fmax3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
           }
-          // 12 + 8 * 6 = 60; the last four
-          m0 = fmax3(m0, __uint_as_float(v[60]), __uint_as_float(v[61]));
-          m1 = fmax3(m1, __uint_as_float(v[62]), __uint_as_float(v[63]));
+          // 12 + 8 * n = EPT - 4; the last four
+          m0 = fmax3(m0, __uint_as_float(v[EPT - 4]), __uint_as_float(v[EPT - 3]));
+          m1 = fmax3(m1, __uint_as_float(v[EPT - 2]), __uint_as_float(v[EPT - 1]));
           mx = fmaxf(fmax3(m0, m1, m2), m3);
         }
         // Row maximum over both halves. The barrier also orders the two halves' S reads before
@@ -900,8 +917,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const bool rescale = (m_new != m_run) && (m_run != -INFINITY);
         const float alpha = rescale ? fast_exp2(m_run - m_new) : 1.f;
         if (j > jb_t && __any_sync(0xffffffffu, rescale)) {
-          // S_t ready implies the previous P_t V product has finished, so O_t is stable here;
-          // each half rescales its own D/2 columns of the row
+          if constexpr (kIndep) {
+            // S(k) is computed ahead of P(k-1) V(k-1) here, so O_t is stable only once that product
+            // has been committed: the release of the V stage it read is the same event
+            const uint32_t kp = tcount - 1u;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_v_empty + 8 * (2 * t + (kp & 1u)), (kp >> 1) & 1u, wctx, kWaitVEmpty));
+            if (!ok) break;
+            tc_fence_after();
+          }
+          // (shared mode: S_t ready implies the previous P_t V product has finished.) Each half
+          // rescales its own D/2 columns of the row.
 #pragma unroll 1
           for (int ch = 0; ch < D / 32; ++ch) {          // rare path: keep it small
             uint32_t ov[16];
@@ -922,9 +947,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint64_t negm2 = pack_f2(__float_as_uint(neg_m), __float_as_uint(neg_m));
         uint64_t sum_a = 0ull, sum_b = 0ull;                 // two packed accumulators
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
+        for (int ch = 0; ch < NCH; ++ch) {
           uint32_t pk[16];
-          if (ch == 0 ? need0 : need1) {
+          if (need[ch]) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
               float p0, p1, p2, p3;
@@ -940,7 +965,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
             for (int i = 0; i < 16; ++i) pk[i] = 0u;
           }
-          tmem_st16(tmem_s + 32 * h + ch * 16, pk);
+          tmem_st16(tmem_sb + (EPT / 2) * h + ch * 16, pk);
         }
         float sum0, sum1, sum2, sum3;
         unpack_f2(sum_a, sum0, sum1);
@@ -949,7 +974,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         l_run += (sum0 + sum2) + (sum1 + sum3);
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bar_p_full + 8 * t);
+        mbar_arrive(bar_p_full + 8 * (2 * t + sbuf));
         ++tcount;
       }
       if (!ok) break;
@@ -1119,7 +1144,8 @@ template <int D, bool kIndep>
 int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
                        const void* k, const void* v, void* o, const void* rope_table, int32_t* device_status,
                        cudaStream_t stream) {
-  using Cfg = AttnCfg<D>;
+  constexpr int BN = kIndep ? kTileNShort : kTileN;
+  using Cfg = AttnCfg<D, BN>;
   CUtensorMap mq, mk, mv, mo;
   int st;
   if ((st = make_map(&mq, q, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;

@@ -212,6 +212,7 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   const bool even_group = (group % 2) == 0;
   const bool independent = mean_key_tiles(n_bins, bin_seg_ptr, seg_start, seg_len) < 8.0;
   const bool pair_rows = !even_group && !independent;
+  const int32_t tile_n = independent ? kTileNShort : kTileN;   // key rows per tile of the chosen mode
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
   TableLayout L;
   L.bin_seg_ptr = kHeaderInts;
@@ -232,7 +233,7 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
       // first key row (rounded down to a key tile) that query tile q0 can see
       auto kv_lo_of = [&](int32_t q0) {
         while (s + 1 < s_hi && seg_start[s + 1] <= q0) ++s;       // segment holding row q0
-        return (seg_start[s] / kTileN) * kTileN;
+        return (seg_start[s] / tile_n) * tile_n;
       };
       const int32_t step = pair_rows ? 2 * kTileM : kTileM;
       for (int32_t q0 = 0; q0 < used; q0 += step) {
@@ -242,18 +243,18 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
         it.q_row0[0] = q0;
         if (!pair_rows) {                       // two heads, same rows
           it.q_row0[1] = q0;
-          it.n_kv_tiles = (std::min(q0 + kTileM, used) - it.kv_row0 + kTileN - 1) / kTileN;
+          it.n_kv_tiles = (std::min(q0 + kTileM, used) - it.kv_row0 + tile_n - 1) / tile_n;
           it.jb1 = 0;
           it.je0 = it.n_kv_tiles;
         } else if (q0 + kTileM < used) {        // two consecutive row tiles
           const int32_t q1 = q0 + kTileM;
           it.q_row0[1] = q1;
-          it.jb1 = (kv_lo_of(q1) - it.kv_row0) / kTileN;
-          it.je0 = (q1 - it.kv_row0) / kTileN;  // slot 0 ends with its diagonal tile
-          it.n_kv_tiles = (std::min(q1 + kTileM, used) - it.kv_row0 + kTileN - 1) / kTileN;
+          it.jb1 = (kv_lo_of(q1) - it.kv_row0) / tile_n;
+          it.je0 = (q1 - it.kv_row0) / tile_n;  // slot 0 ends with its diagonal tile
+          it.n_kv_tiles = (std::min(q1 + kTileM, used) - it.kv_row0 + tile_n - 1) / tile_n;
         } else {                                // last, unpaired row tile of the bin
           it.q_row0[1] = -1;
-          it.n_kv_tiles = (used - it.kv_row0 + kTileN - 1) / kTileN;
+          it.n_kv_tiles = (used - it.kv_row0 + tile_n - 1) / tile_n;
           it.jb1 = it.n_kv_tiles;
           it.je0 = it.n_kv_tiles;
         }

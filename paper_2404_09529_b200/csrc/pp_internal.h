@@ -10,7 +10,8 @@
 namespace pp {
 
 constexpr int kTileM = 128;      // query rows per work item (tcgen05 MMA M)
-constexpr int kTileN = 128;      // key rows per inner step (tcgen05 MMA N of Q.K^T)
+constexpr int kTileN = 128;      // key rows per inner step (tcgen05 MMA N of Q.K^T), shared-stream mode
+constexpr int kTileNShort = 64;  // the same in independent-slot mode (short work items)
 constexpr int kHeaderInts = 16;  // table header, see build_prefill_tables
 constexpr int kHeaderCounter = 10;   // header word the persistent CTAs draw work indices from
 constexpr int kItemInts = 16;
@@ -18,7 +19,7 @@ constexpr int kItemInts = 16;
 // One entry of the attention work list: two query-tile slots sharing one key/value tile stream.
 struct WorkItem {
   int32_t bin;
-  int32_t kv_row0;      // first key row of the stream (multiple of kTileN)
+  int32_t kv_row0;      // first key row of the stream (multiple of the mode's key tile)
   int32_t n_kv_tiles;   // key tiles in the stream
   int32_t q_row0[2];    // first query row of each slot; -1 = slot unused
   int32_t jb1;          // slot 1 takes part in key tiles [jb1, n_kv_tiles)
