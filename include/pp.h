@@ -150,11 +150,6 @@ int pp_prefill_attention(const pp_attn_params* params,
  *   bin_seg_ptr, seg_start, seg_len, seg_prompt, k   host packing arrays from pp_pack
  *   lengths      host [k], original prompt order: rows of each prompt to cache (<= its segment)
  *   q            device [R, M, Hq, D] bf16, raw queries, read only
- *   q_rot        device buffer of the same shape, or NULL. May be q itself. When given and the
- *                prompts are short (work items of a few key tiles), the queries are rotated into it
- *                by a separate pass and the attention kernel reads it, which is faster there than
- *                rotating inside the kernel; otherwise it is left untouched. With NULL the queries
- *                are always rotated on the fly.
  *   k_           device [R, M, Hkv, D] bf16 in/out: overwritten with the rotated keys
  *   v, o         as in pp_prefill_attention
  *   k_cache, v_cache, cache_off, cache_cap   as in pp_unpack_kv (original prompt order)
@@ -162,14 +157,14 @@ int pp_prefill_attention(const pp_attn_params* params,
  *                cos/sin table of capacity * D/2 pairs); host_workspace: host staging of the same
  *                size or at least the table part, pinned memory keeps the call asynchronous
  * params->flags: PP_FLAG_ROPE_ONLY runs only the rotation / unpack kernels, PP_FLAG_SKIP_ROPE only the
- * attention kernel (k_, and q_rot where it is used, hold rotated values already). Outputs are bit-identical to the two-call
- * path. Errors as the two calls it replaces.
+ * attention kernel (k_ holds rotated keys already). Outputs are bit-identical to the two-call path.
+ * Errors as the two calls it replaces.
  */
 size_t pp_prefill_fused_workspace_bytes(const pp_attn_params* params, int32_t k);
 int pp_prefill_fused(const pp_attn_params* params,
                      const int32_t* bin_seg_ptr, const int32_t* seg_start, const int32_t* seg_len,
                      const int32_t* seg_prompt, int32_t k, const int32_t* lengths,
-                     const void* q, void* q_rot, void* k_, const void* v, void* o,
+                     const void* q, void* k_, const void* v, void* o,
                      void* k_cache, void* v_cache, const int64_t* cache_off, const int32_t* cache_cap,
                      void* workspace, void* host_workspace, size_t workspace_bytes,
                      int32_t* device_status, void* stream);

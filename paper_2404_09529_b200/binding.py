@@ -58,7 +58,7 @@ def load_library():
         "pp_prefill_attention": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp,
                                                 ctypes.c_size_t, vp, vp]),
         "pp_prefill_fused_workspace_bytes": (ctypes.c_size_t, [pp, ctypes.c_int32]),
-        "pp_prefill_fused": (ctypes.c_int, [pp, i32p, i32p, i32p, i32p, ctypes.c_int32, i32p, vp, vp, vp, vp, vp, vp, vp,
+        "pp_prefill_fused": (ctypes.c_int, [pp, i32p, i32p, i32p, i32p, ctypes.c_int32, i32p, vp, vp, vp, vp, vp, vp,
                                             i64p, i32p, vp, vp, ctypes.c_size_t, vp, vp]),
         "pp_selftest_bounded_wait": (ctypes.c_int, [vp, ctypes.c_uint32, vp]),
         "pp_unpack_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32]),
@@ -162,14 +162,14 @@ def pp_prefill_fused_workspace_bytes(params: AttnParams, k: int) -> int:
     return int(load_library().pp_prefill_fused_workspace_bytes(ctypes.byref(params), k))
 
 
-def pp_prefill_fused(params: AttnParams, pack: Packing, lengths, q, q_rot, k, v, o, k_cache, v_cache, cache_off,
+def pp_prefill_fused(params: AttnParams, pack: Packing, lengths, q, k, v, o, k_cache, v_cache, cache_off,
                      cache_cap, workspace, host_workspace, workspace_bytes: int, device_status=None,
                      stream: int = 0) -> None:
     l, cc = _i32(lengths), _i32(cache_cap)
     co = np.ascontiguousarray(np.asarray(cache_off, dtype=np.int64))
     st = load_library().pp_prefill_fused(
         ctypes.byref(params), _p32(pack.bin_seg_ptr), _p32(pack.seg_start), _p32(pack.seg_len),
-        _p32(pack.seg_prompt), pack.k, _p32(l), _addr(q), _addr(q_rot), _addr(k), _addr(v), _addr(o), _addr(k_cache),
+        _p32(pack.seg_prompt), pack.k, _p32(l), _addr(q), _addr(k), _addr(v), _addr(o), _addr(k_cache),
         _addr(v_cache), co.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), _p32(cc), _addr(workspace),
         _addr(host_workspace), workspace_bytes, _addr(device_status), stream)
     _check(st, "pp_prefill_fused")

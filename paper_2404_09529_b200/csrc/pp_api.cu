@@ -135,7 +135,7 @@ extern "C" size_t pp_prefill_fused_workspace_bytes(const pp_attn_params* params,
 
 extern "C" int pp_prefill_fused(const pp_attn_params* params, const int32_t* bin_seg_ptr,
                                 const int32_t* seg_start, const int32_t* seg_len, const int32_t* seg_prompt,
-                                int32_t k, const int32_t* lengths, const void* q, void* q_rot, void* k_,
+                                int32_t k, const int32_t* lengths, const void* q, void* k_,
                                 const void* v, void* o, void* k_cache, void* v_cache, const int64_t* cache_off, const int32_t* cache_cap,
                                 void* workspace, void* host_workspace, size_t workspace_bytes,
                                 int32_t* device_status, void* stream) {
@@ -146,7 +146,7 @@ extern "C" int pp_prefill_fused(const pp_attn_params* params, const int32_t* bin
     return PP_ERR_INVALID_ARG;
   st = pp::validate_packing(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k);
   if (st != PP_OK) return st;
-  if (!pp::aligned16(q) || !pp::aligned16(q_rot) || !pp::aligned16(k_) || !pp::aligned16(v) || !pp::aligned16(o) ||
+  if (!pp::aligned16(q) || !pp::aligned16(k_) || !pp::aligned16(v) || !pp::aligned16(o) ||
       !pp::aligned16(k_cache) || !pp::aligned16(v_cache) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return PP_ERR_ALIGNMENT;
   const pp::FusedLayout f = pp::fused_layout(*params, k);
@@ -180,18 +180,9 @@ extern "C" int pp_prefill_fused(const pp_attn_params* params, const int32_t* bin
                                 (int32_t)f.off_cache_off, rope_table, k_, v, k_cache, v_cache, stream);
     if (st != PP_OK) return st;
   }
-  // Short work items: rotating a Q tile inside the attention kernel sits on each item's critical
-  // path, so when the caller offers a buffer for rotated queries, a separate pass writes them there
-  // and the attention kernel reads that buffer. Long items: rotate on the fly, Q is read once.
-  const bool pre_rotate_q = L.independent_slots && q_rot != nullptr;
-  if (pre_rotate_q && !(params->flags & PP_FLAG_SKIP_ROPE)) {
-    pp_attn_params only_q = *params;
-    only_q.n_kv_heads = 0;
-    if ((st = pp::launch_rope(only_q, d_table, L, q, q_rot, nullptr, stream)) != PP_OK) return st;
-  }
   if (params->flags & PP_FLAG_ROPE_ONLY) return PP_OK;
-  return pp::launch_attention(*params, d_table, L, pre_rotate_q ? q_rot : q, k_, v, o,
-                              pre_rotate_q ? nullptr : rope_table, device_status, stream);
+  // the attention kernel rotates every Q tile in shared memory, so Q is read from HBM once
+  return pp::launch_attention(*params, d_table, L, q, k_, v, o, rope_table, device_status, stream);
 }
 
 extern "C" int pp_selftest_bounded_wait(int32_t* device_status, uint32_t limit_ms, void* stream) {

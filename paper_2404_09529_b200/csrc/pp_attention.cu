@@ -758,6 +758,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // kernel, then reports the slot's Q as ready. Waits for the TMA load of Q first.
     auto rotate_q = [&](const int pos, const uint32_t parity) -> bool {
       if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * t, parity, wctx, kWaitQFull))) return false;
+      PROF_LAP(8);
       if (pos > 0) {
         constexpr int kUnits = D / 16;                 // 16-byte units per half of a row
         const uint32_t q_row = s_q + (uint32_t)t * Cfg::kQBytes + (uint32_t)row * 128;
@@ -980,6 +981,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (!ok) break;
 
       if (kIndep && args.rope_table) {
+        PROF_LAP(5);
         // Independent mode, fused path: while this item's last P V product is still running, get the
         // next item's Q ready, so that its first S tile is computed under this item's epilogue.
         const uint32_t nring = (uint32_t)t * kRing + (it_n + 1) % kRing;
@@ -1002,6 +1004,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
           ok = rotate_q(n_pos, (it_n + 1) & 1u);
           if (!ok) break;
+          PROF_LAP(11);
         }
       }
       // epilogue: O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store

@@ -83,19 +83,14 @@ class PrefillBatch:
                            self.ws.unpack_bytes, stream)
         self.ws.release(slot)
 
-    def run_fused(self, repack: bool = False, flags: int = 0, q_rot="scratch") -> None:
-        """One pass of the hot path through the fused entry point (asynchronous). q is left untouched;
-        q_rot: "scratch" = a separate buffer for rotated queries, None = always rotate on the fly."""
-        if q_rot == "scratch":
-            if not hasattr(self, "q_scratch"):
-                self.q_scratch = torch.empty_like(self.q)
-            q_rot = self.q_scratch
+    def run_fused(self, repack: bool = False, flags: int = 0) -> None:
+        """One pass of the hot path through the fused entry point (asynchronous). q is left untouched."""
         if repack:
             self._pack()
         stream = torch.cuda.current_stream().cuda_stream
         _, _, slot = self.ws.acquire()
         self.params.flags = flags
-        B.pp_prefill_fused(self.params, self.pack, self.lengths, self.q, q_rot, self.kk, self.v, self.o, self.k_cache,
+        B.pp_prefill_fused(self.params, self.pack, self.lengths, self.q, self.kk, self.v, self.o, self.k_cache,
                            self.v_cache, self.cache_off, self.cache_cap, self.ws.fused_dev,
                            self.ws.fused_host(slot), self.ws.fused_bytes, self.ws.status, stream)
         self.ws.release(slot)
