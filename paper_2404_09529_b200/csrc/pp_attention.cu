@@ -47,6 +47,8 @@ constexpr int kAttnThreads = 640;
 constexpr int kSoftmaxThreads = 256;       // per slot: two threads per query row
 constexpr uint32_t kTmemCols = 512;
 constexpr int kRegsSoftmax = 104;          // setmaxnreg budgets: 640 threads start with 96 registers each;
+constexpr int kRegsSoftmaxIndep = 120;     // independent mode: 256 softmax threads at 120, 256 helper threads at 88
+constexpr int kRegsHelper = 88;
 constexpr int kRegsOther = 64;              // warps 0-3 give back 32 each, the 512 softmax threads take 8 each
 constexpr uint32_t kRing = 3;               // decoded work items in flight between the fetching thread and its readers
 constexpr int kRingInts = 20;              // ints per ring entry
@@ -107,13 +109,17 @@ struct WaitCtx {
   unsigned long long limit_ns;
 };
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, int code) {
-  const unsigned long long t0 = global_ns();
+  // The clock is read only every 32 failed polls (each poll may park the thread in hardware for a
+  // while), so a short wait costs nothing but the polls; the limit counts from the first reading.
+  unsigned long long t0 = 0;
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 31u) == 0) {
       if (*w.abort_flag) return false;
-      if (global_ns() - t0 > w.limit_ns) {
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > w.limit_ns) {
         *w.abort_flag = 1;
         if (w.status) atomicCAS(w.status, 0, code);
         return false;
@@ -344,7 +350,7 @@ __device__ __forceinline__ void ring_write(volatile int* e, int w, const Work& w
 }
 
 enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWaitKFull, kWaitKEmpty,
-                kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty };
+                kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty, kWaitPair, kWaitEpilogue, kWaitRowSum };
 
 // kIndep = false: the two slots of a CTA work on one item and share its K/V stream (long
 //   sequences, GQA head pairs). kIndep = true: every slot draws its own single-tile items and loads
@@ -388,11 +394,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const uint32_t bar_v_full = s_misc + 320;      // [4]
   const uint32_t bar_v_empty = s_misc + 352;     // [4]
   const uint32_t bar_q_rot = s_misc + 384;       // [2] Q_t has been rotated in place (fused path)
+  const uint32_t bar_pair0 = s_misc + 896;       // [2 slots][4 quadrants] rendezvous of the two warps that share rows
+  const uint32_t bar_epi0 = s_misc + 960;        // [2] rendezvous of a slot's 128 epilogue threads
+  const uint32_t bar_l_ready = s_misc + 976;     // [2] independent mode: the slot's row sums are in shared memory
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 400);
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 404);
   volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 416);   // [2 rings][kRing][kRingInts]
   volatile float* s_xchg = reinterpret_cast<volatile float*>(misc + 1024);   // [2 slots][2 halves][128 rows]
-  static_assert(416 + 2 * kRing * kRingInts * 4 <= 1024, "ring does not fit");
+  static_assert(416 + 2 * kRing * kRingInts * 4 <= 896, "ring does not fit");
   static_assert(NK <= 4 && NV <= 4, "barrier slots");
 
   const int warp = threadIdx.x >> 5;
@@ -409,13 +418,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_q_full + 8 * i, 1);
       mbar_init(bar_q_empty + 8 * i, 1);
-      mbar_init(bar_q_rot + 8 * i, kSoftmaxThreads);
+      mbar_init(bar_q_rot + 8 * i, kIndep ? kSoftmaxThreads / 2 : kSoftmaxThreads);
       for (int b = 0; b < 2; ++b) {
         mbar_init(bar_s_full + 8 * (2 * i + b), 1);
-        mbar_init(bar_p_full + 8 * (2 * i + b), kSoftmaxThreads);
+        mbar_init(bar_p_full + 8 * (2 * i + b), kIndep ? kSoftmaxThreads / 2 : kSoftmaxThreads);
       }
       mbar_init(bar_o_full + 8 * i, 1);
-      mbar_init(bar_o_empty + 8 * i, kSoftmaxThreads / 2);   // the half-0 threads run the epilogue
+      mbar_init(bar_o_empty + 8 * i, kIndep ? kSoftmaxThreads / 2 : kSoftmaxThreads);
+      mbar_init(bar_epi0 + 8 * i, kSoftmaxThreads / 2);
+      mbar_init(bar_l_ready + 8 * i, kSoftmaxThreads / 2);
+      for (int qd = 0; qd < 4; ++qd) mbar_init(bar_pair0 + 8 * (4 * i + qd), 64);
     }
     for (int s = 0; s < NK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
     for (int s = 0; s < NV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
@@ -717,11 +729,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (ok) ok = slot_step(1, j, jb1, je1, tc1);
         }
         if (!ok) break;
-        if (je0 <= 0) {                        // unused slot: keep its per-item barriers in step
+        // Unused slot: keep its per-item barriers in step. o_full must not complete two phases
+        // before every softmax thread has seen the first, so wait until all of them are past the
+        // previous item's o_full (they signal that on o_empty).
+        if (je0 <= 0) {
+          if (!(ok = mbar_wait(bar_o_empty + 0, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
           mbar_arrive(bar_q_empty + 0);
           mbar_arrive(bar_o_full + 0);
         }
         if (jb1 >= je1) {
+          if (!(ok = mbar_wait(bar_o_empty + 8, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
           mbar_arrive(bar_q_empty + 8);
           mbar_arrive(bar_o_full + 8);
         }
@@ -734,20 +751,328 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }   // shared-stream roles
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-    // All softmax warps run the same code (slot and half at run time): the unrolled row loops are
-    // large and several copies of them would not stay resident in the instruction caches.
     const int t = (warp - 4) >> 3;                   // slot
-    const int h = ((warp - 4) >> 2) & 1;             // which 64 keys of a 128-key tile this thread owns
+    const int h = ((warp - 4) >> 2) & 1;             // shared mode: which 64 keys of a 128-key tile this thread owns
     const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
     const int row = quad * 32 + lane;                // query row inside the tile
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const uint32_t tmem_s = tmem_base + Cfg::kTmemS + 128u * t + lane_base;
     const uint32_t tmem_o = tmem_base + Cfg::kTmemO + (uint32_t)D * t + lane_base;
+
+    if constexpr (kIndep) {
+      // ---------------------------------------------------------------- independent mode
+      // Per slot: warps with h == 0 are the softmax threads, one per query row (all 64 scores of a
+      // tile), and never leave the tile loop; warps with h == 1 are helper threads, one per row, which
+      // rotate the next item's Q in shared memory (fused path) and run the epilogue of the previous
+      // item, both off the softmax threads' critical path.
+      const float c_scale = args.scale_log2;
+      const int32_t* tb = args.table;
+      const uint32_t ring0 = (uint32_t)t * kRing;
+      // row sums travel from the softmax thread to the helper of the same row, double-buffered by item
+      volatile float* x_l = s_xchg + t * 128 + row;            // + 256 * (item & 1)
+      bool ok = true;
+      // key range [key_lo, key_hi] of this thread's row from a ring entry (empty for padding rows)
+      auto row_range = [&](const volatile int* e, int& key_lo, int& key_hi) {
+        const int i_row = e[4] + row;
+        key_lo = 1; key_hi = 0;
+        if (i_row < e[12]) {
+          key_lo = e[14];
+          if (!(e[18] & 1)) {                          // several prompts in this tile: walk their starts
+            for (int sg = e[16] + 1; sg < e[13]; ++sg) {
+              const int st = __ldg(tb + args.off_seg_start + sg);
+              if (st > i_row) break;
+              key_lo = st;
+            }
+          }
+          key_hi = i_row;
+        }
+      };
+      if (h == 0) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxIndep));
+        uint32_t it_n = 0, tcount = 0;
+        PROF_DECL(12);
+        while (true) {
+          const uint32_t ring = ring0 + it_n % kRing;
+          PROF_LAP(8);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull));
+          PROF_LAP(0);
+          if (!ok) break;
+          const volatile int* e = s_ring + ring * kRingInts;
+          const int w = e[0], item_kv_row0 = e[2], n_tiles = e[3];
+          int key_lo, key_hi;
+          if (w >= 0) row_range(e, key_lo, key_hi);
+          mbar_arrive(bar_item_empty + 8 * ring);
+          if (w < 0) break;
+          float m_run = -INFINITY;      // running maximum of the row, in scaled log2 units
+          float l_run = 0.f;            // running sum of exp2(s * c - m_run)
+          PROF_LAP(8);
+          for (int j = 0; j < n_tiles; ++j) {
+            constexpr int EPT = BN;                              // scores per thread and tile
+            constexpr int NCH = EPT / 32;                        // 32-column TMEM round trips
+            const int kv0 = item_kv_row0 + j * BN;
+            const int c_lo = max(key_lo - kv0, 0);
+            const int c_hi = min(key_hi - kv0, EPT - 1);         // visible columns [c_lo, c_hi]
+            const bool full = (c_lo == 0) && (c_hi == EPT - 1);
+            const bool warp_full = __all_sync(0xffffffffu, full);
+            bool need[NCH];
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch)
+              need[ch] = __any_sync(0xffffffffu, max(c_lo, 32 * ch) <= min(c_hi, 32 * ch + 31));
+            const uint32_t sbuf = tcount & 1u;                   // tile k of the stream lives in S buffer k & 1
+            const uint32_t tmem_sb = tmem_s + 64u * sbuf;
+            PROF_LAP(5);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * (2 * t + sbuf), (tcount >> 1) & 1u, wctx, kWaitS));
+            if (!ok) break;
+            tc_fence_after();
+            PROF_LAP(1);
+            uint32_t v[EPT];
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+              if (need[ch]) {
+                tmem_ld32(tmem_sb + 32 * ch, *reinterpret_cast<uint32_t(*)[32]>(&v[32 * ch]));
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[32 * ch + i] = 0xff800000u;        // -inf
+              }
+            }
+            tc_wait_ld();
+            PROF_LAP(2);
+            if (!warp_full) {
+              if (__any_sync(0xffffffffu, c_hi < EPT - 1)) {
+#pragma unroll
+                for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
+              }
+              if (__any_sync(0xffffffffu, c_lo > 0)) {
+#pragma unroll
+                for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
+              }
+            }
+            float mx;
+            {
+              float m0 = fmax3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+              float m1 = fmax3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+              float m2 = fmax3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
+              float m3 = fmax3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
+#pragma unroll
+              for (int i = 12; i + 7 < EPT; i += 8) {
+                m0 = fmax3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                m1 = fmax3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                m2 = fmax3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                m3 = fmax3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+              }
+              m0 = fmax3(m0, __uint_as_float(v[EPT - 4]), __uint_as_float(v[EPT - 3]));
+              m1 = fmax3(m1, __uint_as_float(v[EPT - 2]), __uint_as_float(v[EPT - 1]));
+              mx = fmaxf(fmax3(m0, m1, m2), m3);
+            }
+            PROF_LAP(3);
+            // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
+            const float m_tile = mx * c_scale;
+            float m_new = m_run;
+            if (m_tile > m_run + 8.f) m_new = m_tile;
+            const bool rescale = (m_new != m_run) && (m_run != -INFINITY);
+            const float alpha = rescale ? fast_exp2(m_run - m_new) : 1.f;
+            if (j > 0 && __any_sync(0xffffffffu, rescale)) {
+              // S(k) is computed ahead of P(k-1) V(k-1), so O_t is stable only once that product has
+              // been committed: the release of the V stage it read is the same event
+              const uint32_t kp = tcount - 1u;
+              ok = __all_sync(0xffffffffu, mbar_wait(bar_v_empty + 8 * (2 * t + (kp & 1u)), (kp >> 1) & 1u, wctx, kWaitVEmpty));
+              if (!ok) break;
+              tc_fence_after();
+#pragma unroll 1
+              for (int ch = 0; ch < D / 16; ++ch) {          // rare path: keep it small
+                uint32_t ov[16];
+                tmem_ld16(tmem_o + ch * 16, ov);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                tmem_st16(tmem_o + ch * 16, ov);
+              }
+            }
+            PROF_LAP(9);
+            l_run *= alpha;
+            m_run = m_new;
+            const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
+            // p = exp2(s * c - m), row sum, P (bf16) written over the first half of the S buffer
+            const uint64_t c2 = pack_f2(__float_as_uint(c_scale), __float_as_uint(c_scale));
+            const uint64_t negm2 = pack_f2(__float_as_uint(neg_m), __float_as_uint(neg_m));
+            uint64_t sum_a = 0ull, sum_b = 0ull;
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+              uint32_t pk[16];
+              if (need[ch]) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                  float p0, p1, p2, p3;
+                  unpack_f2(fma_f2(pack_f2(v[ch * 32 + i], v[ch * 32 + i + 1]), c2, negm2), p0, p1);
+                  unpack_f2(fma_f2(pack_f2(v[ch * 32 + i + 2], v[ch * 32 + i + 3]), c2, negm2), p2, p3);
+                  p0 = fast_exp2(p0); p1 = fast_exp2(p1); p2 = fast_exp2(p2); p3 = fast_exp2(p3);
+                  sum_a = add_f2(sum_a, pack_f2(__float_as_uint(p0), __float_as_uint(p1)));
+                  sum_b = add_f2(sum_b, pack_f2(__float_as_uint(p2), __float_as_uint(p3)));
+                  pk[i >> 1] = pack_bf16(p0, p1);
+                  pk[(i >> 1) + 1] = pack_bf16(p2, p3);
+                }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pk[i] = 0u;
+              }
+              // S(k) was read completely above, so P(k) may overwrite its first columns
+              tmem_st16(tmem_sb + ch * 16, pk);
+            }
+            float sum0, sum1, sum2, sum3;
+            unpack_f2(sum_a, sum0, sum1);
+            unpack_f2(sum_b, sum2, sum3);
+            PROF_LAP(4);
+            l_run += (sum0 + sum2) + (sum1 + sum3);
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p_full + 8 * (2 * t + sbuf));
+            ++tcount;
+          }
+          if (!ok) break;
+          // hand the row sum to the helper thread of this row (arrive has release semantics)
+          x_l[256 * (it_n & 1u)] = l_run;
+          mbar_arrive(bar_l_ready + 8 * t);
+          PROF_LAP(7);
+          ++it_n;
+        }
+#ifdef PP_PROFILE
+        prof_acc[10] = tcount;
+        if (row == 0) PROF_STORE(8 + 12 * t, 12);
+#endif
+      } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsHelper));
+        const uint32_t bar_epi = bar_epi0 + 8 * (uint32_t)t;
+        uint32_t epi_ph = 0;
+        auto rendezvous = [&](const uint32_t bar, uint32_t& ph, const int code) -> bool {
+          mbar_arrive(bar);
+          const bool r = __all_sync(0xffffffffu, mbar_wait(bar, ph, wctx, code));
+          ph ^= 1u;
+          return r;
+        };
+        uint32_t it_n = 0;
+        int p_q_row0 = 0, p_head = 0, p_bin = 0;         // coordinates of the previous item (its epilogue is due)
+        while (true) {
+          const uint32_t ring = ring0 + it_n % kRing;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull));
+          if (!ok) break;
+          const volatile int* e = s_ring + ring * kRingInts;
+          const int w = e[0], c_bin = e[1], c_q_row0 = e[4], c_head = e[9];
+          int key_lo = 1, key_hi = 0;
+          if (w >= 0 && args.rope_table) row_range(e, key_lo, key_hi);
+          mbar_arrive(bar_item_empty + 8 * ring);
+          if (w >= 0 && args.rope_table) {
+            // rotate row `row` of this item's Q in shared memory by the angles of its position, with
+            // the same fp32 arithmetic and rounding as the stand-alone kernel, then report Q_t ready
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * t, it_n & 1u, wctx, kWaitQFull));
+            if (!ok) break;
+            const int pos = key_hi - key_lo;             // < 0 for padding rows
+            if (pos > 0) {
+              constexpr int kUnits = D / 16;             // 16-byte (lower, upper) unit pairs per row
+              const uint32_t q_row = s_q + (uint32_t)t * Cfg::kQBytes + (uint32_t)row * 128;
+              // table[g][pos] = (cos, sin) of j = 2g and 2g + 1: consecutive rows read consecutive 16 bytes
+              const float4* tab = reinterpret_cast<const float4*>(args.rope_table) + pos;
+#pragma unroll 1
+              for (int u0 = 0; u0 < kUnits; u0 += 2) {
+                float4 cs[2][4];                         // table loads of two units first: one L2 round trip
+#pragma unroll
+                for (int uu = 0; uu < 2; ++uu)
+#pragma unroll
+                  for (int i = 0; i < 4; ++i)
+                    cs[uu][i] = __ldg(tab + (size_t)((u0 + uu) * 4 + i) * (size_t)args.capacity);
+#pragma unroll
+                for (int uu = 0; uu < 2; ++uu) {
+                  const int u = u0 + uu;                 // pairs (8u .. 8u+7, + D/2)
+                  const uint32_t a_lo = q_row + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4);
+                  const uint32_t a_hi = (D == 128)
+                      ? q_row + (BM * 128) + ((((uint32_t)u) ^ ((uint32_t)row & 7u)) << 4)
+                      : q_row + ((((uint32_t)(u + kUnits)) ^ ((uint32_t)row & 7u)) << 4);
+                  uint32_t lo[4], hi[4];
+                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo[0]), "=r"(lo[1]), "=r"(lo[2]), "=r"(lo[3]) : "r"(a_lo));
+                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi[0]), "=r"(hi[1]), "=r"(hi[2]), "=r"(hi[3]) : "r"(a_hi));
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    const float4 c = cs[uu][i];          // (cos, sin) of two consecutive j
+                    const __nv_bfloat162 l2 = *reinterpret_cast<__nv_bfloat162*>(&lo[i]);
+                    const __nv_bfloat162 h2 = *reinterpret_cast<__nv_bfloat162*>(&hi[i]);
+                    const float2 a = __bfloat1622float2(l2), b = __bfloat1622float2(h2);
+                    lo[i] = pack_bf16(__fmaf_rn(a.x, c.x, -__fmul_rn(b.x, c.y)), __fmaf_rn(a.y, c.z, -__fmul_rn(b.y, c.w)));
+                    hi[i] = pack_bf16(__fmaf_rn(b.x, c.x, __fmul_rn(a.x, c.y)), __fmaf_rn(b.y, c.z, __fmul_rn(a.y, c.w)));
+                  }
+                  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_lo), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+                  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_hi), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+                }
+              }
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
+            }
+            mbar_arrive(bar_q_rot + 8 * t);
+          }
+          if (it_n > 0) {
+            // epilogue of the previous item: O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store
+            const uint32_t pi = it_n - 1u;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full + 8 * t, pi & 1u, wctx, kWaitOFull));
+            if (!ok) break;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_l_ready + 8 * t, pi & 1u, wctx, kWaitRowSum));
+            if (!ok) break;
+            tc_fence_after();
+            const float l_row = x_l[256 * (pi & 1u)];
+            const float inv_l = l_row > 0.f ? 1.f / l_row : 0.f;
+            const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes;
+            const uint32_t stage_row = stage + (uint32_t)row * 128;
+#pragma unroll 1
+            for (int hh = 0; hh < D / 64; ++hh) {          // 64 columns (one TMA box) at a time
+              // the staging buffer is free once the previous store has read it
+              if (row == 0) tma_store_wait_read();
+              if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
+              uint32_t ov[64];
+              tmem_ld32(tmem_o + hh * 64, *reinterpret_cast<uint32_t(*)[32]>(&ov[0]));
+              tmem_ld32(tmem_o + hh * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[32]));
+              tc_wait_ld();
+              if (hh == D / 64 - 1) {
+                tc_fence_before();
+                mbar_arrive(bar_o_empty + 8 * t);        // O_t may be overwritten by the next item now
+              }
+#pragma unroll
+              for (int c16 = 0; c16 < 8; ++c16) {
+                const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)row & 7u)) << 4);
+                const uint32_t w0 = pack_bf16(__uint_as_float(ov[c16 * 8 + 0]) * inv_l, __uint_as_float(ov[c16 * 8 + 1]) * inv_l);
+                const uint32_t w1 = pack_bf16(__uint_as_float(ov[c16 * 8 + 2]) * inv_l, __uint_as_float(ov[c16 * 8 + 3]) * inv_l);
+                const uint32_t w2 = pack_bf16(__uint_as_float(ov[c16 * 8 + 4]) * inv_l, __uint_as_float(ov[c16 * 8 + 5]) * inv_l);
+                const uint32_t w3 = pack_bf16(__uint_as_float(ov[c16 * 8 + 6]) * inv_l, __uint_as_float(ov[c16 * 8 + 7]) * inv_l);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+              }
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
+              if (row == 0) {
+                tma_store_4d(&map_o, stage, hh * 64, p_head, p_q_row0, p_bin);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+              }
+            }
+            if (!ok) break;
+          }
+          if (w < 0) break;
+          p_q_row0 = c_q_row0; p_head = c_head; p_bin = c_bin;
+          ++it_n;
+        }
+        if (row == 0) tma_store_wait_read();     // staging must outlive the last store's read
+      }
+    } else {
+    // ---------------------------------------------------------------- shared-stream mode
+    // All softmax warps run the same code (slot and half at run time): the unrolled row loops are
+    // large and several copies of them would not stay resident in the instruction caches.
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     volatile float* x_mine = s_xchg + (t * 2 + h) * 128 + row;
     volatile float* x_other = s_xchg + (t * 2 + (h ^ 1)) * 128 + row;
-    const int bar_pair = 1 + t * 4 + quad;           // named barrier of the two warps that share these rows
-    const int bar_epi = 9 + t;                       // named barrier of the slot's 128 half-0 threads
+    // Rendezvous points are mbarriers (arrive, then a bounded wait) rather than named barriers, so
+    // that a warp whose partner gave up on a wait cannot be left waiting for it.
+    const uint32_t bar_pair = bar_pair0 + 8 * (uint32_t)(t * 4 + quad);
+    const uint32_t bar_epi = bar_epi0 + 8 * (uint32_t)t;
+    uint32_t pair_ph = 0, epi_ph = 0;
+    auto rendezvous = [&](const uint32_t bar, uint32_t& ph, const int code) -> bool {
+      mbar_arrive(bar);
+      const bool r = __all_sync(0xffffffffu, mbar_wait(bar, ph, wctx, code));
+      ph ^= 1u;
+      return r;
+    };
     const float c_scale = args.scale_log2;
     const int32_t* tb = args.table;
     uint32_t it_n = 0, tcount = 0;
@@ -908,7 +1233,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // Row maximum over both halves. The barrier also orders the two halves' S reads before
         // either writes P over the S columns.
         *x_mine = mx;
-        asm volatile("bar.sync %0, 64;" ::"r"(bar_pair) : "memory");
+        if (!(ok = rendezvous(bar_pair, pair_ph, kWaitPair))) break;
         mx = fmaxf(mx, *x_other);
         PROF_LAP(3);
         // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
@@ -1016,9 +1341,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // the half-1 threads hand their share of the row sum to the half-0 threads, which run the
         // epilogue; the second barrier keeps the exchange slot from being reused too early
         if (h == 1) *x_mine = l_run;
-        asm volatile("bar.sync %0, 64;" ::"r"(bar_pair) : "memory");
+        if (!(ok = rendezvous(bar_pair, pair_ph, kWaitPair))) break;
         const float l_row = (h == 0) ? l_run + *x_other : 0.f;
-        asm volatile("bar.sync %0, 64;" ::"r"(bar_pair) : "memory");
+        if (!(ok = rendezvous(bar_pair, pair_ph, kWaitPair))) break;
+        if (h == 1) mbar_arrive(bar_o_empty + 8 * t);      // this thread is past o_full and never reads O_t
         if (h == 0) {
           tc_fence_after();
           const float inv_l = l_row > 0.f ? 1.f / l_row : 0.f;
@@ -1028,7 +1354,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int hh = 0; hh < D / 64; ++hh) {          // 64 columns (one TMA box) at a time
             // the staging buffer is free once the previous store has read it
             if (row == 0) tma_store_wait_read();
-            asm volatile("bar.sync %0, %1;" ::"r"(bar_epi), "n"(kSoftmaxThreads / 2) : "memory");
+            if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
             uint32_t ov[64];
             tmem_ld32(tmem_o + hh * 64, *reinterpret_cast<uint32_t(*)[32]>(&ov[0]));
             tmem_ld32(tmem_o + hh * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[32]));
@@ -1047,16 +1373,17 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("bar.sync %0, %1;" ::"r"(bar_epi), "n"(kSoftmaxThreads / 2) : "memory");
+            if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
             if (row == 0) {
               tma_store_4d(&map_o, stage, hh * 64, head_t, q_row0_t, item_bin);
               asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
           }
         }
-      } else if (h == 0) {
+      } else {
         mbar_arrive(bar_o_empty + 8 * t);
       }
+      if (!ok) break;
       PROF_LAP(7);
       ++it_n;
     }
@@ -1065,6 +1392,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     prof_acc[10] = tcount;
     if (row == 0 && h == 0) PROF_STORE(8 + 12 * t, 12);
 #endif
+    }   // shared-stream mode
   }
 
   tc_fence_before();

@@ -144,6 +144,9 @@ struct SegExt {                    // per-segment arrays appended to the prefill
   int32_t off_true_len, off_cap, off_cache_off;   // int32 offsets into the table (cache_off: int64 data)
 };
 
+constexpr int kRuRows = 8;   // packed rows per block of the fused K/V kernel
+constexpr int kRuV = 8;      // 16-byte V copies in flight per thread
+constexpr int kRuK = 2;      // (lower, upper) K pairs in flight per thread
 template <int D>
 __global__ void __launch_bounds__(kRopeThreads)
 rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
@@ -154,14 +157,14 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
   constexpr int kHalf = D / 2;
   constexpr int kPairUnits = kHalf / 8;             // (lower, upper) 16-byte pairs per head
   constexpr int kVecs = D / 8;                      // 16-byte vectors per head
-  __shared__ int32_t s_pos[kRopeRows];              // restart position, -1 for padding rows
-  __shared__ int64_t s_dst[kRopeRows];              // cache element offset of (head 0, this position); -1: not cached
-  __shared__ int64_t s_head_stride[kRopeRows];      // cache_cap * D
+  __shared__ int32_t s_pos[kRuRows];              // restart position, -1 for padding rows
+  __shared__ int64_t s_dst[kRuRows];              // cache element offset of (head 0, this position); -1: not cached
+  __shared__ int64_t s_head_stride[kRuRows];      // cache_cap * D
 
-  const int64_t row0 = (int64_t)blockIdx.x * kRopeRows;
+  const int64_t row0 = (int64_t)blockIdx.x * kRuRows;
   const int64_t n_rows = (int64_t)n_bins * capacity;
   const int tid = threadIdx.x;
-  if (tid < kRopeRows) {
+  if (tid < kRuRows) {
     const int64_t row = row0 + tid;
     int32_t pos = -1;
     int64_t dst = -1, stride = 0;
@@ -190,14 +193,14 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
 
   // V rows first: plain 16-byte copies, four in flight per thread
   const int units_v = n_kv_heads * kVecs;
-  for (int u0 = tid; u0 < kRopeRows * units_v; u0 += 4 * kRopeThreads) {
-    uint4 val[4];
-    int64_t dsts[4];
+  for (int u0 = tid; u0 < kRuRows * units_v; u0 += kRuV * kRopeThreads) {
+    uint4 val[kRuV];
+    int64_t dsts[kRuV];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kRuV; ++i) {
       const int u = u0 + i * kRopeThreads;
       dsts[i] = -1;
-      if (u < kRopeRows * units_v) {
+      if (u < kRuRows * units_v) {
         const int r = u / units_v, w = u - r * units_v;
         if (s_dst[r] >= 0) {
           const int head = w / kVecs, c = w - head * kVecs;
@@ -207,19 +210,19 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
       }
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < kRuV; ++i)
       if (dsts[i] >= 0) *reinterpret_cast<uint4*>(v_cache + dsts[i]) = val[i];
   }
   // K rows: rotate, write back to the packed tensor and into the cache; two pairs in flight
   const int units_k = n_kv_heads * kPairUnits;
-  for (int u0 = tid; u0 < kRopeRows * units_k; u0 += 2 * kRopeThreads) {
-    uint4 lo[2], hi[2];
-    int rr[2], hh[2], cc[2];
+  for (int u0 = tid; u0 < kRuRows * units_k; u0 += kRuK * kRopeThreads) {
+    uint4 lo[kRuK], hi[kRuK];
+    int rr[kRuK], hh[kRuK], cc[kRuK];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kRuK; ++i) {
       const int u = u0 + i * kRopeThreads;
       rr[i] = -1;
-      if (u < kRopeRows * units_k) {
+      if (u < kRuRows * units_k) {
         const int r = u / units_k, w = u - r * units_k;
         if (s_pos[r] >= 0) {
           rr[i] = r; hh[i] = w / kPairUnits; cc[i] = w - hh[i] * kPairUnits;
@@ -230,7 +233,7 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
       }
     }
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kRuK; ++i) {
       if (rr[i] < 0) continue;
       const int r = rr[i], head = hh[i], c = cc[i];
       const int32_t pos = s_pos[r];
@@ -280,7 +283,7 @@ int launch_rope_unpack(const pp_attn_params& p, const int32_t* d_table, const Ta
                        int32_t off_true_len, int32_t off_cap, int32_t off_cache_off, const void* rope_table,
                        void* k, const void* v, void* k_cache, void* v_cache, void* stream) {
   const int64_t n_rows = (int64_t)p.n_bins * p.capacity;
-  const unsigned grid = (unsigned)((n_rows + kRopeRows - 1) / kRopeRows);
+  const unsigned grid = (unsigned)((n_rows + kRuRows - 1) / kRuRows);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const SegExt ext{off_true_len, off_cap, off_cache_off};
   if (p.head_dim == 128) {
