@@ -34,7 +34,7 @@ DEFAULT_WORKLOAD = "llama2_7b"
 # DRAM traffic of one attention-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu capture summarised in profiles/attention_llama2_7b.md; None where no capture exists for
 # the workload.
-NCU_ATTENTION_TRAFFIC_BYTES = {"llama2_7b": 562.1e6}
+NCU_ATTENTION_TRAFFIC_BYTES = {"llama2_7b": 563.9e6}
 
 
 def load_peaks():
@@ -412,7 +412,7 @@ def main():
                        "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
                        "rope_base": cfg.rope_base, "path": path, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                        "l2": f"no flush: each step streams {resident_mb:.0f} MB of tensors, larger than the 126 MB L2"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": (3 if path == "three_call" else 4) * args.steps, "roofline": roofline,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "kernels": kernels, "padded": padded,
             "routes": {"three_call": {"tokens_per_s": whole_job_tokens_per_s(world, T, route_ms["three_call"]),
                                       "ms_per_step": route_ms["three_call"],

@@ -15,19 +15,23 @@
 //   warp 1       issues tcgen05.mma: S_t = Q_t K^T into TMEM, O_t += P_t V with P_t read from TMEM;
 //                the two slots alternate so that one slot's MMAs run while the other's softmax works
 //   warps 2-3    TMA-load Q of slot 0 / slot 1
+//   warps 4-11   softmax and epilogue of slot 0: two threads per query row (TMEM lane = row), one per
+//                64-key half of a tile; the row maximum is exchanged through shared memory
+//   warps 12-19  the same for slot 1
 // Independent mode (short items). Every slot draws its own items (one query tile each) and walks
 // their 64-row key tiles on its own; S_t has two 64-column buffers so that the scores of tile k+1
-// and the product P(k) V(k) are computed while the softmax threads work.
+// and the product P(k) V(k) are computed while the softmax threads work on tile k.
 //   warps 0-1    issue the tcgen05.mma of slot 0 / slot 1
 //   warps 2-3    draw items and TMA-load Q, K, V of slot 0 / slot 1 (two K and two V stages each)
-// Both modes:
-//   warps 4-11   softmax of slot 0: two threads per query row (TMEM lane = row), one per half tile
-//   warps 12-19  softmax of slot 1
-// Softmax: tcgen05.ld the thread's scores, mask to the row's key range, row maximum exchanged
-// between the two halves through shared memory, lazy running maximum (O is rescaled only when
-// the maximum grows by more than 2^8), exp2, P written as bf16 over the S columns; at the end of
-// an item O / l goes through a swizzled staging buffer and a TMA store.
-// TMEM: S0 | S1 | O0 | O1 = 512 columns. Every mbarrier wait is bounded.
+//   warps 4-7    softmax threads of slot 0, one per query row; they never leave the tile loop
+//   warps 8-11   helper threads of slot 0, one per row: rotate the next item's Q in shared memory
+//                (fused path) and run the previous item's epilogue
+//   warps 12-19  the same for slot 1
+// Softmax: tcgen05.ld the thread's scores, mask to the row's key range, lazy running maximum (O is
+// rescaled only when the maximum grows by more than 2^8), exp2, P written as bf16 over the S
+// columns. Epilogue: O / l goes through a swizzled staging buffer and a TMA store.
+// TMEM: S0 | S1 | O0 | O1 = 512 columns. Every wait is an mbarrier wait with a time limit, also the
+// rendezvous between warps (no named barriers), so a failed wait ends the kernel with a status code.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <cuda_bf16.h>
