@@ -304,6 +304,23 @@ def main():
     value = whole_job_tokens_per_s(world, T, ms_per_step)
     batch.load(q_tok, k_tok, v_tok)
 
+    # ---------------------------------------------------------------- host share of a step (rank-local)
+    import time as _time
+    t0 = _time.perf_counter()
+    for _ in range(50):
+        pp.pp_pack(lengths, 0)
+    pack_us = (_time.perf_counter() - t0) / 50 * 1e6
+    enqueue_us = 0.0
+    for _ in range(20):
+        torch.cuda.synchronize()                 # idle device: the call returns as soon as it has enqueued
+        t0 = _time.perf_counter()
+        routes[path]()
+        enqueue_us += (_time.perf_counter() - t0) / 20 * 1e6     # pack + table build + copies + launches
+    torch.cuda.synchronize()
+    host = {"pp_pack_us": pack_us, "enqueue_us_per_step": enqueue_us,
+            "note": "host time to pack and enqueue one step; it overlaps the previous step's kernels"}
+    batch.load(q_tok, k_tok, v_tok)
+
     # ---------------------------------------------------------------- per-kernel times (rank-local)
     n_it = args.kernel_iters
     ms_rope = time_loop(lambda: batch.run(flags=pp.PP_FLAG_ROPE_ONLY, unpack=False), n_it)
@@ -365,6 +382,18 @@ def main():
                   "attention_speedup_packed_vs_padded": ms_pad_attn / dom["ms"]}
         del pb
         torch.cuda.empty_cache()
+        # one prompt per bin with its true length: masking and tile skipping without the packing
+        vb = PrefillBatch(lengths, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, mode="varlen")
+        vb.load(q_tok, k_tok, v_tok)
+        if path == "fused":
+            ms_var = time_loop(lambda: vb.run_fused(), n_pad)
+        else:
+            ms_var = time_loop(lambda: vb.run(), n_pad)
+        padded["unpacked_varlen"] = {"tokens_per_s": T / (ms_var * 1e-3), "ms_per_step": ms_var,
+                                     "rows_allocated": int(vb.pack.n_bins) * int(vb.pack.capacity),
+                                     "speedup_packed_vs_unpacked_varlen": ms_var / ms_per_step}
+        del vb
+        torch.cuda.empty_cache()
 
     # ---------------------------------------------------------------- end to end from host buffers
     params = pp.AttnParams(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base, 0.0, 0, 0, 0)
@@ -413,7 +442,7 @@ def main():
                        "rope_base": cfg.rope_base, "path": path, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                        "l2": f"no flush: each step streams {resident_mb:.0f} MB of tensors, larger than the 126 MB L2"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roofline,
-            "cpu_baseline": cpu_baseline, "kernels": kernels, "padded": padded,
+            "cpu_baseline": cpu_baseline, "host": host, "kernels": kernels, "padded": padded,
             "routes": {"three_call": {"tokens_per_s": whole_job_tokens_per_s(world, T, route_ms["three_call"]),
                                       "ms_per_step": route_ms["three_call"],
                                       "api": "pp_pack + pp_prefill_attention + pp_unpack_kv"},

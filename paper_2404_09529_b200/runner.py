@@ -16,6 +16,8 @@ class PrefillBatch:
     mode "padded": the full-batching baseline -- one bin per prompt in original order, every
     bin declared as a single segment of the full capacity, so all k*m rows are computed;
     unpack still copies only each prompt's true rows.
+    mode "varlen": one bin per prompt in original order, each declared with its true length: the
+    mask and tile skipping without the bin packing (isolates what packing adds).
     """
 
     def __init__(self, lengths, n_q_heads: int, n_kv_heads: int, head_dim: int, rope_base: float,
@@ -57,6 +59,13 @@ class PrefillBatch:
             self.pack = B.pp_pack(np.full(self.k, m, dtype=np.int32), 0)
             self.bin_of = np.arange(self.k, dtype=np.int32)
             self.off_of = np.zeros(self.k, dtype=np.int32)
+        elif self.mode == "varlen":
+            m = int(self.lengths.max())
+            ar = np.arange(self.k, dtype=np.int32)
+            self.pack = B.Packing(self.k, m, np.arange(self.k + 1, dtype=np.int32), ar.copy(),
+                                  np.zeros(self.k, np.int32), self.lengths.copy(), ar.copy(),
+                                  np.zeros(self.k, np.int32))
+            self.bin_of, self.off_of = self.pack.bin_of, self.pack.off_of
         else:
             raise ValueError(self.mode)
         self.params = B.AttnParams(self.hq, self.hkv, self.d, self.rope_base, self.softmax_scale,

@@ -221,3 +221,27 @@ def test_fused_large_configs_sampled_parity(name):
     prompts = sorted(set(int(order[i]) for i in (0, len(order) // 2, -1)))
     compare_sampled(b, lengths, q.cpu(), k.cpu(), v.cpu(), cfg.rope_base, prompts=prompts,
                     kv_heads=[0, cfg.n_kv_heads - 1], n_rows=32)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,route", [("llama2_7b", "fused"), ("llama2_7b", "three_call"),
+                                        ("many_short", "fused"), ("llama3_8b_gqa", "three_call")])
+def test_repeated_runs_are_bit_identical_and_clean(name, route):
+    """The persistent kernel draws work from a counter, so the tile-to-CTA assignment differs from
+    run to run; the results must not (every output element is written by exactly one thread in a
+    fixed arithmetic order), and no wait may ever give up."""
+    from paper_2404_09529_b200.runner import PrefillBatch
+    cfg, lengths, q, k, v = _workload(name)
+    b = PrefillBatch(lengths, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.rope_base)
+    ref = None
+    for it in range(12):
+        b.load(q, k, v)                      # K (and Q on the three-call route) are rotated in place
+        b.run_fused() if route == "fused" else b.run()
+        torch.cuda.synchronize()
+        assert b.device_status() == 0, (name, route, it)
+        got = (b.o_tokens().clone(), b.k_cache.clone(), b.v_cache.clone())
+        if ref is None:
+            ref = got
+        else:
+            for a, c in zip(ref, got):
+                assert torch.equal(a, c), (name, route, it)
