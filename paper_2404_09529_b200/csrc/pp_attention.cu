@@ -1401,6 +1401,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   tc_fence_before();
   __syncthreads();
+  if (*s_abort) {
+    // A wait gave up: TMA loads and MMAs of this CTA may still be in flight. Give them time to land
+    // (they take microseconds) before shared memory and TMEM are handed back.
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 100000ull) {}
+    __syncthreads();
+  }
   if (warp == 0) {
     __syncwarp();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -1456,10 +1463,14 @@ int make_map(CUtensorMap* map, const void* ptr, int64_t R, int64_t M, int64_t H,
 }
 
 unsigned long long wait_limit_ns() {
-  // Debug override of the device-side wait limit, in milliseconds.
+  // Debug overrides of the device-side wait limit, in milliseconds or microseconds.
   if (const char* e = std::getenv("PP_WAIT_LIMIT_MS")) {
     const long ms = std::atol(e);
     if (ms > 0) return (unsigned long long)ms * 1000000ull;
+  }
+  if (const char* e = std::getenv("PP_WAIT_LIMIT_US")) {
+    const long us = std::atol(e);
+    if (us > 0) return (unsigned long long)us * 1000ull;
   }
   return 2000000000ull;   // 2 s
 }
