@@ -239,7 +239,11 @@ int pp_unpack_kv_static(const pp_attn_params* params,
  *                            lengths), laid out [Hkv, lengths[i], D]
  *   arena, arena_bytes       device scratch >= pp_prefill_host_arena_bytes(params, lengths, k),
  *                            256-byte aligned
- * Pinned host buffers give full copy bandwidth; pageable ones work too.
+ * Pinned host buffers give full copy bandwidth; pageable ones work too. When the prompts are
+ * large (>= 1 MB of Q, K, V each on average) the bins are cut into up to four groups that are
+ * pipelined over streams the library creates once per device and thread, so that the uploads of
+ * one group overlap the kernels and downloads of the others; the call still returns only when
+ * everything is on the host, and work already queued on `stream` is waited for first.
  * Errors: as the three calls it is made of, plus PP_ERR_DEVICE_TIMEOUT.
  */
 size_t pp_prefill_host_arena_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k);

@@ -2,6 +2,7 @@
 // Algorithm 1 lines 5-8 of the prepacking paper; see include/pp.h for the contracts.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -254,8 +255,10 @@ namespace {
 
 size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
 
+constexpr int kHostGroups = 4;     // groups of bins pp_prefill_host pipelines over its own streams
+
 struct ArenaPlan {
-  size_t q, k, v, o, kc, vc, ws_attn, ws_unpack, status, total;
+  size_t q, k, v, o, kc, vc, ws_attn, ws_attn_stride, ws_unpack, ws_unpack_stride, status, total;
 };
 
 ArenaPlan plan_arena(const pp_attn_params& p, int32_t n_bins, int32_t capacity, int64_t total_tokens, int32_t k) {
@@ -270,11 +273,41 @@ ArenaPlan plan_arena(const pp_attn_params& p, int32_t n_bins, int32_t capacity, 
   a.o = off; off += up256(qb);
   a.kc = off; off += up256(cb);
   a.vc = off; off += up256(cb);
-  a.ws_attn = off; off += up256(sizeof(int32_t) * prefill_table_ints(n_bins, capacity, k));
-  a.ws_unpack = off; off += up256(unpack_table_bytes(k));
+  // one table workspace per group (each sized for the whole batch: they are small)
+  a.ws_attn_stride = up256(sizeof(int32_t) * prefill_table_ints(n_bins, capacity, k));
+  a.ws_attn = off; off += kHostGroups * a.ws_attn_stride;
+  a.ws_unpack_stride = up256(unpack_table_bytes(k));
+  a.ws_unpack = off; off += kHostGroups * a.ws_unpack_stride;
   a.status = off; off += 256;
   a.total = off;
   return a;
+}
+
+// Streams and events pp_prefill_host pipelines over, created on first use per device.
+struct HostPipe {
+  cudaStream_t stream[kHostGroups] = {};
+  cudaEvent_t done[kHostGroups] = {};
+  cudaEvent_t start = nullptr;
+  int device = -1;
+};
+int host_pipe(HostPipe** out) {
+  static thread_local HostPipe pipe;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return note_cuda_error((int)e, "cudaGetDevice");
+  if (pipe.device != dev) {
+    for (int g = 0; g < kHostGroups; ++g) {
+      if ((e = cudaStreamCreateWithFlags(&pipe.stream[g], cudaStreamNonBlocking)) != cudaSuccess)
+        return note_cuda_error((int)e, "cudaStreamCreate");
+      if ((e = cudaEventCreateWithFlags(&pipe.done[g], cudaEventDisableTiming)) != cudaSuccess)
+        return note_cuda_error((int)e, "cudaEventCreate");
+    }
+    if ((e = cudaEventCreateWithFlags(&pipe.start, cudaEventDisableTiming)) != cudaSuccess)
+      return note_cuda_error((int)e, "cudaEventCreate");
+    pipe.device = dev;
+  }
+  *out = &pipe;
+  return PP_OK;
 }
 
 }  // namespace
@@ -323,38 +356,87 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
     const size_t kv_row = (size_t)params->n_kv_heads * params->head_dim * 2;
     cudaError_t e;
 #define PP_TRY(call, what) do { e = (call); if (e != cudaSuccess) return pp::note_cuda_error((int)e, what); } while (0)
-    // TENSORIZE: zero the packed buffers (padding rows must be finite), then one copy per prompt
-    PP_TRY(cudaMemsetAsync(base + a.q, 0, a.o - a.q, s), "memset packed q/k/v");
+    // The bins are cut into up to kHostGroups groups, each with its own stream: uploads of one group
+    // overlap the kernels of another and the downloads of a third (PCIe is full duplex), instead of
+    // all uploads, then all kernels, then all downloads.
+    pp::HostPipe* pipe = nullptr;
+    if ((st = pp::host_pipe(&pipe)) != PP_OK) return st;
+    // Only worth it when the per-prompt copies are large: with many small prompts the copies are
+    // latency-bound and one stream with two large cache downloads is faster.
+    const size_t mean_prompt_bytes = (size_t)(total / k) * (q_row + 2 * kv_row);
+    const int n_groups = mean_prompt_bytes >= (size_t(1) << 20) ? std::min<int>(pp::kHostGroups, r) : 1;
     PP_TRY(cudaMemsetAsync(base + a.status, 0, 4, s), "memset status");
-    for (int32_t i = 0; i < k; ++i) {
-      const size_t row = (size_t)bin_of[i] * cap + off_of[i];
-      PP_TRY(cudaMemcpyAsync(base + a.q + row * q_row, (const char*)q_host + tok_off[i] * q_row,
-                             lengths[i] * q_row, cudaMemcpyHostToDevice, s), "H2D q");
-      PP_TRY(cudaMemcpyAsync(base + a.k + row * kv_row, (const char*)k_host + tok_off[i] * kv_row,
-                             lengths[i] * kv_row, cudaMemcpyHostToDevice, s), "H2D k");
-      PP_TRY(cudaMemcpyAsync(base + a.v + row * kv_row, (const char*)v_host + tok_off[i] * kv_row,
-                             lengths[i] * kv_row, cudaMemcpyHostToDevice, s), "H2D v");
-    }
-    // host staging for the two tables (pageable: the copies below stage them before returning)
-    std::vector<int32_t> h_ws_attn(pp::prefill_table_ints(r, cap, k));
-    std::vector<int64_t> h_ws_unpack((pp::unpack_table_bytes(k) + 7) / 8);
-    st = pp_prefill_attention(params, bin_seg_ptr.data(), seg_start.data(), seg_len.data(), k, base + a.q,
-                              base + a.k, base + a.v, base + a.o, base + a.ws_attn, h_ws_attn.data(),
-                              h_ws_attn.size() * sizeof(int32_t),
-                              reinterpret_cast<int32_t*>(base + a.status), stream);
-    if (st != PP_OK) return st;
-    st = pp_unpack_kv(params, bin_of.data(), off_of.data(), lengths, k, base + a.k, base + a.v, base + a.kc,
-                      base + a.vc, cache_off.data(), lengths, base + a.ws_unpack, h_ws_unpack.data(),
-                      h_ws_unpack.size() * 8, stream);
-    if (st != PP_OK) return st;
-    // UNPACK to the host: caches are already in original order; O goes back prompt by prompt
-    const size_t cache_bytes = (size_t)total * kv_row;
-    PP_TRY(cudaMemcpyAsync(k_cache_host, base + a.kc, cache_bytes, cudaMemcpyDeviceToHost, s), "D2H k cache");
-    PP_TRY(cudaMemcpyAsync(v_cache_host, base + a.vc, cache_bytes, cudaMemcpyDeviceToHost, s), "D2H v cache");
-    for (int32_t i = 0; i < k; ++i) {
-      const size_t row = (size_t)bin_of[i] * cap + off_of[i];
-      PP_TRY(cudaMemcpyAsync((char*)o_host + tok_off[i] * q_row, base + a.o + row * q_row, lengths[i] * q_row,
-                             cudaMemcpyDeviceToHost, s), "D2H o");
+    PP_TRY(cudaEventRecord(pipe->start, s), "event record");
+    // host staging for the tables of every group (pageable: the copies stage them before returning)
+    std::vector<std::vector<int32_t>> h_ws_attn(n_groups);
+    std::vector<std::vector<int64_t>> h_ws_unpack(n_groups);
+    std::vector<int32_t> g_ptr, g_bin_of, g_off_of, g_len, g_ids;
+    std::vector<int64_t> g_cache_off;
+    for (int g = 0; g < n_groups; ++g) {
+      const int32_t b0 = (int32_t)((int64_t)r * g / n_groups), b1 = (int32_t)((int64_t)r * (g + 1) / n_groups);
+      const int32_t s0 = bin_seg_ptr[b0], s1 = bin_seg_ptr[b1], kg = s1 - s0;
+      cudaStream_t sg = pipe->stream[g];
+      PP_TRY(cudaStreamWaitEvent(sg, pipe->start, 0), "stream wait");
+      // TENSORIZE: zero the group's packed rows (padding rows must be finite), then one copy per prompt
+      const size_t rows0 = (size_t)b0 * cap, nrows = (size_t)(b1 - b0) * cap;
+      PP_TRY(cudaMemsetAsync(base + a.q + rows0 * q_row, 0, nrows * q_row, sg), "memset packed q");
+      PP_TRY(cudaMemsetAsync(base + a.k + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed k");
+      PP_TRY(cudaMemsetAsync(base + a.v + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed v");
+      g_ptr.assign(bin_seg_ptr.begin() + b0, bin_seg_ptr.begin() + b1 + 1);
+      for (int32_t& x : g_ptr) x -= s0;
+      g_ids.assign(seg_prompt.begin() + s0, seg_prompt.begin() + s1);       // the group's prompts
+      g_bin_of.resize(kg); g_off_of.resize(kg); g_len.resize(kg); g_cache_off.resize(kg);
+      for (int32_t j = 0; j < kg; ++j) {
+        const int32_t i = g_ids[j];
+        g_bin_of[j] = bin_of[i] - b0;
+        g_off_of[j] = off_of[i];
+        g_len[j] = lengths[i];
+        g_cache_off[j] = cache_off[i];
+        const size_t row = (size_t)bin_of[i] * cap + off_of[i];
+        PP_TRY(cudaMemcpyAsync(base + a.q + row * q_row, (const char*)q_host + tok_off[i] * q_row,
+                               lengths[i] * q_row, cudaMemcpyHostToDevice, sg), "H2D q");
+        PP_TRY(cudaMemcpyAsync(base + a.k + row * kv_row, (const char*)k_host + tok_off[i] * kv_row,
+                               lengths[i] * kv_row, cudaMemcpyHostToDevice, sg), "H2D k");
+        PP_TRY(cudaMemcpyAsync(base + a.v + row * kv_row, (const char*)v_host + tok_off[i] * kv_row,
+                               lengths[i] * kv_row, cudaMemcpyHostToDevice, sg), "H2D v");
+      }
+      pp_attn_params gp = *params;
+      gp.n_bins = b1 - b0;
+      h_ws_attn[g].resize(pp::prefill_table_ints(gp.n_bins, cap, kg));
+      h_ws_unpack[g].resize((pp::unpack_table_bytes(kg) + 7) / 8);
+      st = pp_prefill_attention(&gp, g_ptr.data(), seg_start.data() + s0, seg_len.data() + s0, kg,
+                                base + a.q + rows0 * q_row, base + a.k + rows0 * kv_row, base + a.v + rows0 * kv_row,
+                                base + a.o + rows0 * q_row, base + a.ws_attn + g * a.ws_attn_stride,
+                                h_ws_attn[g].data(), h_ws_attn[g].size() * sizeof(int32_t),
+                                reinterpret_cast<int32_t*>(base + a.status), sg);
+      if (st != PP_OK) return st;
+      st = pp_unpack_kv(&gp, g_bin_of.data(), g_off_of.data(), g_len.data(), kg, base + a.k + rows0 * kv_row,
+                        base + a.v + rows0 * kv_row, base + a.kc, base + a.vc, g_cache_off.data(), g_len.data(),
+                        base + a.ws_unpack + g * a.ws_unpack_stride, h_ws_unpack[g].data(),
+                        h_ws_unpack[g].size() * 8, sg);
+      if (st != PP_OK) return st;
+      // UNPACK to the host, prompt by prompt (caches and O are in original order there); a single
+      // group takes the caches in two large copies instead
+      if (n_groups == 1) {
+        const size_t cache_bytes = (size_t)total * kv_row;
+        PP_TRY(cudaMemcpyAsync(k_cache_host, base + a.kc, cache_bytes, cudaMemcpyDeviceToHost, sg), "D2H k cache");
+        PP_TRY(cudaMemcpyAsync(v_cache_host, base + a.vc, cache_bytes, cudaMemcpyDeviceToHost, sg), "D2H v cache");
+      }
+      for (int32_t j = 0; j < kg; ++j) {
+        const int32_t i = g_ids[j];
+        const size_t row = (size_t)bin_of[i] * cap + off_of[i];
+        const size_t cbytes = (size_t)lengths[i] * kv_row;
+        if (n_groups > 1) {
+          PP_TRY(cudaMemcpyAsync((char*)k_cache_host + cache_off[i] * 2, base + a.kc + cache_off[i] * 2, cbytes,
+                                 cudaMemcpyDeviceToHost, sg), "D2H k cache");
+          PP_TRY(cudaMemcpyAsync((char*)v_cache_host + cache_off[i] * 2, base + a.vc + cache_off[i] * 2, cbytes,
+                                 cudaMemcpyDeviceToHost, sg), "D2H v cache");
+        }
+        PP_TRY(cudaMemcpyAsync((char*)o_host + tok_off[i] * q_row, base + a.o + row * q_row, lengths[i] * q_row,
+                               cudaMemcpyDeviceToHost, sg), "D2H o");
+      }
+      PP_TRY(cudaEventRecord(pipe->done[g], sg), "event record");
+      PP_TRY(cudaStreamWaitEvent(s, pipe->done[g], 0), "stream wait");
     }
     int32_t status = 0;
     PP_TRY(cudaMemcpyAsync(&status, base + a.status, 4, cudaMemcpyDeviceToHost, s), "D2H status");

@@ -162,6 +162,31 @@ def test_host_buffer_entry_point_matches_device_path():
     assert torch.equal(kc, ref.k_cache.cpu()) and torch.equal(vc, ref.v_cache.cpu())
 
 
+def test_host_buffer_entry_point_pipelined_groups():
+    """Large prompts make pp_prefill_host cut the bins into groups that it pipelines over its own
+    streams; the kernels of a group see fewer bins, so O may differ from the whole-batch run only
+    through the tile-to-CTA schedule (it does not: same tiles, same arithmetic) and the caches never."""
+    import paper_2404_09529_b200 as pp
+    lengths = np.array([900, 850, 700, 640, 512, 400, 333, 300, 128, 90, 60, 7], np.int32)
+    hq, hkv, d, base = 8, 2, 128, 500000.0
+    q, k, v = _random_case(lengths, hq, hkv, d, seed=5)
+    ref = run_cuda(lengths, q, k, v, hq, hkv, d, base)
+    params = pp.AttnParams(hq, hkv, d, base, 0.0, 0, 0, 0)
+    nbytes = pp.pp_prefill_host_arena_bytes(params, lengths)
+    arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    qh, kh, vh = (t.contiguous().pin_memory() for t in (q, k, v))
+    o = torch.empty_like(q).pin_memory()
+    kc = torch.empty(k.numel(), dtype=torch.bfloat16).pin_memory()
+    vc = torch.empty(v.numel(), dtype=torch.bfloat16).pin_memory()
+    for _ in range(2):
+        o.zero_(); kc.zero_(); vc.zero_()
+        pp.pp_prefill_host(params, lengths, qh, kh, vh, o, kc, vc, arena, nbytes,
+                           torch.cuda.current_stream().cuda_stream)
+        assert params.n_bins >= 4                      # several groups
+        assert torch.equal(kc, ref.k_cache.cpu()) and torch.equal(vc, ref.v_cache.cpu())
+        assert torch.equal(o, ref.o_tokens().cpu())
+
+
 def test_bounded_wait_gives_up_and_reports():
     """A device-side wait that nothing satisfies returns a status instead of hanging; the context
     stays usable afterwards."""
