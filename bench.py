@@ -420,7 +420,7 @@ def main():
     d2h = (ho.numel() + hkc.numel() + hvc.numel()) * 2
     e2e = {"value": whole_job_tokens_per_s(world, T, ms_e2e / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
-           "api": "pp_prefill_host (pinned host buffers, one H2D copy per prompt and tensor, groups of bins pipelined)"}
+           "api": "pp_prefill_host (pinned host buffers, contiguous copies, groups of prompts pipelined over streams)"}
 
     # ---------------------------------------------------------------- CPU baseline: the oracle as it stands
     cpu_baseline = None

@@ -226,10 +226,10 @@ int pp_unpack_kv_static(const pp_attn_params* params,
 
 /*
  * Whole path from host memory (Algorithm 1 lines 2-8 for one attention layer), for callers whose
- * tensors live on the host. Packs `lengths` (pp_pack, capacity = longest prompt), lays the
- * prompts out as the packed batch on the device (TENSORIZE: one H2D copy per prompt and tensor,
- * padding rows zeroed), runs pp_prefill_attention and pp_unpack_kv there, copies the outputs
- * back and synchronises `stream` before returning.
+ * tensors live on the host. Every tensor goes up in large contiguous copies, is laid out as the
+ * packed batch by a device kernel (TENSORIZE, padding rows zeroed), pp_prefill_attention and
+ * pp_unpack_kv run there, O is gathered back into token order and the outputs are copied back;
+ * `stream` is synchronised before the call returns.
  *   params                   n_q_heads, n_kv_heads, head_dim, rope_base, softmax_scale are
  *                            read; capacity and n_bins are filled in from the packing
  *   q_host                   host bf16 [T, Hq, D], tokens of prompt 0, then prompt 1, ...
@@ -239,11 +239,14 @@ int pp_unpack_kv_static(const pp_attn_params* params,
  *                            lengths), laid out [Hkv, lengths[i], D]
  *   arena, arena_bytes       device scratch >= pp_prefill_host_arena_bytes(params, lengths, k),
  *                            256-byte aligned
- * Pinned host buffers give full copy bandwidth; pageable ones work too. When the prompts are
- * large (>= 1 MB of Q, K, V each on average) the bins are cut into up to four groups that are
- * pipelined over streams the library creates once per device and thread, so that the uploads of
- * one group overlap the kernels and downloads of the others; the call still returns only when
- * everything is on the host, and work already queued on `stream` is waited for first.
+ * Pinned host buffers give full copy bandwidth; pageable ones work too. A batch of 32 MB or more
+ * is cut into up to eight groups of consecutive prompts with about equal token counts. Each
+ * group is packed on its own (pp_pack with the batch-wide capacity = longest prompt; n_bins is the
+ * sum over the groups) and runs on a stream the library creates once per device and thread, so
+ * the uploads of one group overlap the kernels of another and the downloads of a third. Smaller
+ * batches are one group, packed exactly as pp_pack packs the whole batch. The caches do not depend
+ * on the grouping; O depends on it only through the position of tile boundaries (summation
+ * order). Work already queued on `stream` is waited for first.
  * Errors: as the three calls it is made of, plus PP_ERR_DEVICE_TIMEOUT.
  */
 size_t pp_prefill_host_arena_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k);

@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -23,6 +24,12 @@ int note_cuda_error(int cuda_error, const char* what) {
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Internal flag bits (not part of the public header), used by pp_prefill_host to put the small table
+// uploads in front of its large data uploads: a table upload that is queued behind another
+// stream's bulk copy would hold its kernels back for milliseconds.
+constexpr int kFlagUploadOnly = 0x100;     // build and upload the tables, launch nothing
+constexpr int kFlagTablesReady = 0x200;    // the tables are in the workspace already: do not upload
 
 int check_params(const pp_attn_params* p) {
   if (!p) return PP_ERR_INVALID_ARG;
@@ -87,9 +94,12 @@ extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t*
                                 static_cast<int32_t*>(host_workspace), workspace_bytes / sizeof(int32_t), &L);
   if (st != PP_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * (size_t)L.total_ints,
-                                  cudaMemcpyHostToDevice, s);
-  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
+  if (!(flags & pp::kFlagTablesReady)) {
+    cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * (size_t)L.total_ints,
+                                    cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
+  }
+  if (flags & pp::kFlagUploadOnly) return PP_OK;
   int32_t* d_table = static_cast<int32_t*>(workspace);
   if (do_rope) {
     st = pp::launch_rope(*params, d_table, L, q, q, k_, stream);
@@ -240,9 +250,12 @@ extern "C" int pp_unpack_kv(const pp_attn_params* params, const int32_t* bin_of,
     h_coff[i] = cache_off[i];
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, pp::unpack_table_bytes(k),
-                                  cudaMemcpyHostToDevice, s);
-  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "unpack table upload");
+  if (!(params->flags & pp::kFlagTablesReady)) {
+    cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, pp::unpack_table_bytes(k),
+                                    cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return pp::note_cuda_error((int)e, "unpack table upload");
+  }
+  if (params->flags & pp::kFlagUploadOnly) return PP_OK;
   return pp::launch_unpack(*params, static_cast<const int32_t*>(workspace), k, total, k_rot, v, k_cache,
                            v_cache, stream);
 }
@@ -255,32 +268,90 @@ namespace {
 
 size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
 
-constexpr int kHostGroups = 4;     // groups of bins pp_prefill_host pipelines over its own streams
+constexpr int kHostGroups = 8;     // groups of prompts pp_prefill_host pipelines over its own streams
 
-struct ArenaPlan {
-  size_t q, k, v, o, kc, vc, ws_attn, ws_attn_stride, ws_unpack, ws_unpack_stride, status, total;
+// How pp_prefill_host cuts a batch: contiguous ranges of prompts (original order) with about equal
+// token counts, each packed on its own with the batch-wide capacity, so that every tensor of a
+// group is one contiguous range on the host.
+struct HostGroup {
+  int32_t i0 = 0, i1 = 0;          // prompts [i0, i1)
+  int64_t t0 = 0, t1 = 0;          // tokens [t0, t1)
+  int32_t bin0 = 0, n_bins = 0;    // bins [bin0, bin0 + n_bins) of the packed buffers
+  std::vector<int32_t> bin_seg_ptr, seg_prompt, seg_start, seg_len, bin_of, off_of;
+};
+struct HostPlan {
+  int32_t capacity = 0, n_bins = 0;
+  int64_t total_tokens = 0;
+  std::vector<HostGroup> groups;
+  // arena offsets (bytes)
+  size_t q = 0, k = 0, v = 0, o = 0, q_tok = 0, k_tok = 0, v_tok = 0, o_tok = 0, kc = 0, vc = 0;
+  size_t ws_attn = 0, ws_attn_stride = 0, ws_unpack = 0, ws_unpack_stride = 0, map = 0, map_stride = 0;
+  size_t status = 0, total = 0;
 };
 
-ArenaPlan plan_arena(const pp_attn_params& p, int32_t n_bins, int32_t capacity, int64_t total_tokens, int32_t k) {
-  ArenaPlan a{};
-  const size_t rows = (size_t)n_bins * capacity;
-  const size_t qb = rows * p.n_q_heads * p.head_dim * 2, kb = rows * p.n_kv_heads * p.head_dim * 2;
-  const size_t cb = (size_t)total_tokens * p.n_kv_heads * p.head_dim * 2;
+int plan_host(const pp_attn_params& p, const int32_t* lengths, int32_t k, HostPlan* out) {
+  HostPlan& h = *out;
+  int32_t m = 0;
+  for (int32_t i = 0; i < k; ++i) {
+    if (lengths[i] < 1) return PP_ERR_LENGTH;
+    m = std::max(m, lengths[i]);
+    h.total_tokens += lengths[i];
+  }
+  h.capacity = m;
+  const size_t q_row = (size_t)p.n_q_heads * p.head_dim * 2, kv_row = (size_t)p.n_kv_heads * p.head_dim * 2;
+  // pipelining pays once the transfers are tens of megabytes; small batches stay in one group
+  const size_t batch_bytes = (size_t)h.total_tokens * (q_row + 2 * kv_row);
+  int n_groups = batch_bytes >= (size_t(32) << 20) ? std::min<int32_t>(kHostGroups, k) : 1;
+  if (const char* ev = std::getenv("PP_HOST_GROUPS")) {            // debug override
+    const int want = std::atoi(ev);
+    if (want >= 1) n_groups = std::min<int>(std::min<int>(want, kHostGroups), k);
+  }
+  h.groups.resize(n_groups);
+  int32_t i = 0;
+  int64_t t = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    HostGroup& G = h.groups[g];
+    G.i0 = i;
+    G.t0 = t;
+    const int64_t target = h.total_tokens * (g + 1) / n_groups;
+    // at least one prompt per group, and leave at least one for each group after this one
+    while (i < k - (n_groups - 1 - g) && (i == G.i0 || t + lengths[i] <= target || g == n_groups - 1)) t += lengths[i++];
+    G.i1 = i;
+    G.t1 = t;
+    const int32_t kg = G.i1 - G.i0;
+    G.bin_seg_ptr.resize(kg + 1); G.seg_prompt.resize(kg); G.seg_start.resize(kg); G.seg_len.resize(kg);
+    G.bin_of.resize(kg); G.off_of.resize(kg);
+    int32_t r = 0, cap = 0;
+    const int st = pp_pack(lengths + G.i0, kg, m, &r, &cap, G.bin_seg_ptr.data(), G.seg_prompt.data(),
+                           G.seg_start.data(), G.seg_len.data(), G.bin_of.data(), G.off_of.data());
+    if (st != PP_OK) return st;
+    G.bin0 = h.n_bins;
+    G.n_bins = r;
+    h.n_bins += r;
+  }
+  const size_t rows = (size_t)h.n_bins * m;
+  const size_t T = (size_t)h.total_tokens;
   size_t off = 0;
-  a.q = off; off += up256(qb);
-  a.k = off; off += up256(kb);
-  a.v = off; off += up256(kb);
-  a.o = off; off += up256(qb);
-  a.kc = off; off += up256(cb);
-  a.vc = off; off += up256(cb);
-  // one table workspace per group (each sized for the whole batch: they are small)
-  a.ws_attn_stride = up256(sizeof(int32_t) * prefill_table_ints(n_bins, capacity, k));
-  a.ws_attn = off; off += kHostGroups * a.ws_attn_stride;
-  a.ws_unpack_stride = up256(unpack_table_bytes(k));
-  a.ws_unpack = off; off += kHostGroups * a.ws_unpack_stride;
-  a.status = off; off += 256;
-  a.total = off;
-  return a;
+  h.q = off; off += up256(rows * q_row);
+  h.k = off; off += up256(rows * kv_row);
+  h.v = off; off += up256(rows * kv_row);
+  h.o = off; off += up256(rows * q_row);
+  h.q_tok = off; off += up256(T * q_row);
+  h.k_tok = off; off += up256(T * kv_row);
+  h.v_tok = off; off += up256(T * kv_row);
+  h.o_tok = off; off += up256(T * q_row);
+  h.kc = off; off += up256(T * kv_row);
+  h.vc = off; off += up256(T * kv_row);
+  // per-group tables, each sized for the whole batch (they are small)
+  h.ws_attn_stride = up256(sizeof(int32_t) * prefill_table_ints(h.n_bins, m, k));
+  h.ws_attn = off; off += n_groups * h.ws_attn_stride;
+  h.ws_unpack_stride = up256(unpack_table_bytes(k));
+  h.ws_unpack = off; off += n_groups * h.ws_unpack_stride;
+  h.map_stride = up256(sizeof(int64_t) * (2 * (size_t)k + 1));
+  h.map = off; off += n_groups * h.map_stride;
+  h.status = off; off += 256;
+  h.total = off;
+  return PP_OK;
 }
 
 // Streams and events pp_prefill_host pipelines over, created on first use per device.
@@ -288,8 +359,25 @@ struct HostPipe {
   cudaStream_t stream[kHostGroups] = {};
   cudaEvent_t done[kHostGroups] = {};
   cudaEvent_t start = nullptr;
+  void* staging[kHostGroups] = {};        // pinned host staging for each group's tables
+  size_t staging_bytes[kHostGroups] = {};
   int device = -1;
 };
+// Pinned staging of at least `bytes` for group g (kept and grown across calls; every call ends with a
+// synchronize, so a buffer is never reused while a copy still reads it).
+int host_staging(HostPipe* pipe, int g, size_t bytes, void** out) {
+  if (pipe->staging_bytes[g] < bytes) {
+    if (pipe->staging[g]) cudaFreeHost(pipe->staging[g]);
+    pipe->staging[g] = nullptr;
+    pipe->staging_bytes[g] = 0;
+    const size_t want = (bytes + (size_t(1) << 16)) & ~((size_t(1) << 16) - 1);
+    const cudaError_t e = cudaHostAlloc(&pipe->staging[g], want, cudaHostAllocDefault);
+    if (e != cudaSuccess) return note_cuda_error((int)e, "cudaHostAlloc");
+    pipe->staging_bytes[g] = want;
+  }
+  *out = pipe->staging[g];
+  return PP_OK;
+}
 int host_pipe(HostPipe** out) {
   static thread_local HostPipe pipe;
   int dev = 0;
@@ -316,11 +404,14 @@ int host_pipe(HostPipe** out) {
 extern "C" size_t pp_prefill_host_arena_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k) {
   if (!params || !lengths || k < 1) return 0;
   if (params->head_dim != 64 && params->head_dim != 128) return 0;
-  int32_t r = 0, cap = 0;
-  if (pp_pack(lengths, k, 0, &r, &cap, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr) != PP_OK) return 0;
-  int64_t total = 0;
-  for (int32_t i = 0; i < k; ++i) total += lengths[i];
-  return pp::plan_arena(*params, r, cap, total, k).total;
+  if (params->n_q_heads < 1 || params->n_kv_heads < 1) return 0;
+  try {
+    pp::HostPlan h;
+    if (pp::plan_host(*params, lengths, k, &h) != PP_OK) return 0;
+    return h.total;
+  } catch (const std::bad_alloc&) {
+    return 0;
+  }
 }
 
 extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, int32_t k,
@@ -331,116 +422,128 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
       !v_cache_host || !arena)
     return PP_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(arena) & 255u) return PP_ERR_ALIGNMENT;
+  if (params->head_dim != 64 && params->head_dim != 128) return PP_ERR_UNSUPPORTED;
+  if (params->n_q_heads < 1 || params->n_kv_heads < 1) return PP_ERR_INVALID_ARG;
   try {
-    std::vector<int32_t> bin_seg_ptr(k + 1), seg_prompt(k), seg_start(k), seg_len(k), bin_of(k), off_of(k);
-    int32_t r = 0, cap = 0;
-    int st = pp_pack(lengths, k, 0, &r, &cap, bin_seg_ptr.data(), seg_prompt.data(), seg_start.data(),
-                     seg_len.data(), bin_of.data(), off_of.data());
+    pp::HostPlan h;
+    int st = pp::plan_host(*params, lengths, k, &h);
     if (st != PP_OK) return st;
-    params->capacity = cap;
-    params->n_bins = r;
+    params->capacity = h.capacity;
+    params->n_bins = h.n_bins;
     params->flags = 0;
     if ((st = pp::check_params(params)) != PP_OK) return st;
-    int64_t total = 0;
-    std::vector<int64_t> tok_off(k), cache_off(k);
-    for (int32_t i = 0; i < k; ++i) {
-      tok_off[i] = total;
-      cache_off[i] = total * params->n_kv_heads * params->head_dim;
-      total += lengths[i];
-    }
-    const pp::ArenaPlan a = pp::plan_arena(*params, r, cap, total, k);
-    if (arena_bytes < a.total) return PP_ERR_BUFFER_TOO_SMALL;
+    if (arena_bytes < h.total) return PP_ERR_BUFFER_TOO_SMALL;
     char* base = static_cast<char*>(arena);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int32_t cap = h.capacity;
     const size_t q_row = (size_t)params->n_q_heads * params->head_dim * 2;
     const size_t kv_row = (size_t)params->n_kv_heads * params->head_dim * 2;
     cudaError_t e;
 #define PP_TRY(call, what) do { e = (call); if (e != cudaSuccess) return pp::note_cuda_error((int)e, what); } while (0)
-    // The bins are cut into up to kHostGroups groups, each with its own stream: uploads of one group
-    // overlap the kernels of another and the downloads of a third (PCIe is full duplex), instead of
-    // all uploads, then all kernels, then all downloads.
+    // Every group runs on its own stream: one upload per tensor, TENSORIZE on the device, the three
+    // kernels of the path, O gathered back to token order, one download per tensor. The uploads of
+    // one group overlap the kernels of another and the downloads of a third (PCIe is full duplex).
     pp::HostPipe* pipe = nullptr;
     if ((st = pp::host_pipe(&pipe)) != PP_OK) return st;
-    // Only worth it when the per-prompt copies are large: with many small prompts the copies are
-    // latency-bound and one stream with two large cache downloads is faster.
-    const size_t mean_prompt_bytes = (size_t)(total / k) * (q_row + 2 * kv_row);
-    const int n_groups = mean_prompt_bytes >= (size_t(1) << 20) ? std::min<int>(pp::kHostGroups, r) : 1;
-    PP_TRY(cudaMemsetAsync(base + a.status, 0, 4, s), "memset status");
+    const int n_groups = (int)h.groups.size();
+    PP_TRY(cudaMemsetAsync(base + h.status, 0, 4, s), "memset status");
     PP_TRY(cudaEventRecord(pipe->start, s), "event record");
-    // host staging for the tables of every group (pageable: the copies stage them before returning)
-    std::vector<std::vector<int32_t>> h_ws_attn(n_groups);
-    std::vector<std::vector<int64_t>> h_ws_unpack(n_groups);
-    std::vector<int32_t> g_ptr, g_bin_of, g_off_of, g_len, g_ids;
     std::vector<int64_t> g_cache_off;
+    const bool trace = std::getenv("PP_HOST_TRACE") != nullptr;      // debug: print each group's timeline
+    std::vector<cudaEvent_t> tev;
+    auto mark = [&](cudaStream_t st_) { if (trace) { cudaEvent_t ev; cudaEventCreate(&ev); cudaEventRecord(ev, st_); tev.push_back(ev); } };
+    mark(s);
     for (int g = 0; g < n_groups; ++g) {
-      const int32_t b0 = (int32_t)((int64_t)r * g / n_groups), b1 = (int32_t)((int64_t)r * (g + 1) / n_groups);
-      const int32_t s0 = bin_seg_ptr[b0], s1 = bin_seg_ptr[b1], kg = s1 - s0;
+      const pp::HostGroup& G = h.groups[g];
+      const int32_t kg = G.i1 - G.i0;
+      const size_t tok0 = (size_t)G.t0, ntok = (size_t)(G.t1 - G.t0);
+      const size_t rows0 = (size_t)G.bin0 * cap, nrows = (size_t)G.n_bins * cap;
       cudaStream_t sg = pipe->stream[g];
       PP_TRY(cudaStreamWaitEvent(sg, pipe->start, 0), "stream wait");
-      // TENSORIZE: zero the group's packed rows (padding rows must be finite), then one copy per prompt
-      const size_t rows0 = (size_t)b0 * cap, nrows = (size_t)(b1 - b0) * cap;
-      PP_TRY(cudaMemsetAsync(base + a.q + rows0 * q_row, 0, nrows * q_row, sg), "memset packed q");
-      PP_TRY(cudaMemsetAsync(base + a.k + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed k");
-      PP_TRY(cudaMemsetAsync(base + a.v + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed v");
-      g_ptr.assign(bin_seg_ptr.begin() + b0, bin_seg_ptr.begin() + b1 + 1);
-      for (int32_t& x : g_ptr) x -= s0;
-      g_ids.assign(seg_prompt.begin() + s0, seg_prompt.begin() + s1);       // the group's prompts
-      g_bin_of.resize(kg); g_off_of.resize(kg); g_len.resize(kg); g_cache_off.resize(kg);
+      // The small uploads first (token -> packed row map and the two tables of the group, from pinned
+      // staging): queued behind another group's bulk copies they would hold this group's kernels back.
+      const size_t map_bytes = (sizeof(int64_t) * (2 * (size_t)kg + 1) + 255) & ~size_t(255);
+      const size_t attn_tab = (sizeof(int32_t) * pp::prefill_table_ints(G.n_bins, cap, kg) + 255) & ~size_t(255);
+      const size_t unpack_tab = (pp::unpack_table_bytes(kg) + 255) & ~size_t(255);
+      void* stage = nullptr;
+      if ((st = pp::host_staging(pipe, g, map_bytes + attn_tab + unpack_tab, &stage)) != PP_OK) return st;
+      int64_t* map = static_cast<int64_t*>(stage);
+      g_cache_off.resize(kg);
+      int64_t t = 0;
       for (int32_t j = 0; j < kg; ++j) {
-        const int32_t i = g_ids[j];
-        g_bin_of[j] = bin_of[i] - b0;
-        g_off_of[j] = off_of[i];
-        g_len[j] = lengths[i];
-        g_cache_off[j] = cache_off[i];
-        const size_t row = (size_t)bin_of[i] * cap + off_of[i];
-        PP_TRY(cudaMemcpyAsync(base + a.q + row * q_row, (const char*)q_host + tok_off[i] * q_row,
-                               lengths[i] * q_row, cudaMemcpyHostToDevice, sg), "H2D q");
-        PP_TRY(cudaMemcpyAsync(base + a.k + row * kv_row, (const char*)k_host + tok_off[i] * kv_row,
-                               lengths[i] * kv_row, cudaMemcpyHostToDevice, sg), "H2D k");
-        PP_TRY(cudaMemcpyAsync(base + a.v + row * kv_row, (const char*)v_host + tok_off[i] * kv_row,
-                               lengths[i] * kv_row, cudaMemcpyHostToDevice, sg), "H2D v");
+        map[j] = t;
+        map[kg + 1 + j] = (int64_t)G.bin_of[j] * cap + G.off_of[j];
+        g_cache_off[j] = (int64_t)(tok0 + (size_t)t) * params->n_kv_heads * params->head_dim;
+        t += lengths[G.i0 + j];
       }
+      map[kg] = t;
+      int64_t* d_map = reinterpret_cast<int64_t*>(base + h.map + g * h.map_stride);
+      PP_TRY(cudaMemcpyAsync(d_map, map, sizeof(int64_t) * (2 * (size_t)kg + 1), cudaMemcpyHostToDevice, sg), "H2D map");
+      char* gq = base + h.q + rows0 * q_row;
+      char* gk = base + h.k + rows0 * kv_row;
+      char* gv = base + h.v + rows0 * kv_row;
+      char* go = base + h.o + rows0 * q_row;
       pp_attn_params gp = *params;
-      gp.n_bins = b1 - b0;
-      h_ws_attn[g].resize(pp::prefill_table_ints(gp.n_bins, cap, kg));
-      h_ws_unpack[g].resize((pp::unpack_table_bytes(kg) + 7) / 8);
-      st = pp_prefill_attention(&gp, g_ptr.data(), seg_start.data() + s0, seg_len.data() + s0, kg,
-                                base + a.q + rows0 * q_row, base + a.k + rows0 * kv_row, base + a.v + rows0 * kv_row,
-                                base + a.o + rows0 * q_row, base + a.ws_attn + g * a.ws_attn_stride,
-                                h_ws_attn[g].data(), h_ws_attn[g].size() * sizeof(int32_t),
-                                reinterpret_cast<int32_t*>(base + a.status), sg);
+      gp.n_bins = G.n_bins;
+      gp.flags = pp::kFlagUploadOnly;
+      st = pp_prefill_attention(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), kg, gq, gk, gv, go,
+                                base + h.ws_attn + g * h.ws_attn_stride, static_cast<char*>(stage) + map_bytes, attn_tab,
+                                reinterpret_cast<int32_t*>(base + h.status), sg);
       if (st != PP_OK) return st;
-      st = pp_unpack_kv(&gp, g_bin_of.data(), g_off_of.data(), g_len.data(), kg, base + a.k + rows0 * kv_row,
-                        base + a.v + rows0 * kv_row, base + a.kc, base + a.vc, g_cache_off.data(), g_len.data(),
-                        base + a.ws_unpack + g * a.ws_unpack_stride, h_ws_unpack[g].data(),
-                        h_ws_unpack[g].size() * 8, sg);
+      st = pp_unpack_kv(&gp, G.bin_of.data(), G.off_of.data(), lengths + G.i0, kg, gk, gv, base + h.kc, base + h.vc,
+                        g_cache_off.data(), lengths + G.i0, base + h.ws_unpack + g * h.ws_unpack_stride,
+                        static_cast<char*>(stage) + map_bytes + attn_tab, unpack_tab, sg);
       if (st != PP_OK) return st;
-      // UNPACK to the host, prompt by prompt (caches and O are in original order there); a single
-      // group takes the caches in two large copies instead
-      if (n_groups == 1) {
-        const size_t cache_bytes = (size_t)total * kv_row;
-        PP_TRY(cudaMemcpyAsync(k_cache_host, base + a.kc, cache_bytes, cudaMemcpyDeviceToHost, sg), "D2H k cache");
-        PP_TRY(cudaMemcpyAsync(v_cache_host, base + a.vc, cache_bytes, cudaMemcpyDeviceToHost, sg), "D2H v cache");
-      }
-      for (int32_t j = 0; j < kg; ++j) {
-        const int32_t i = g_ids[j];
-        const size_t row = (size_t)bin_of[i] * cap + off_of[i];
-        const size_t cbytes = (size_t)lengths[i] * kv_row;
-        if (n_groups > 1) {
-          PP_TRY(cudaMemcpyAsync((char*)k_cache_host + cache_off[i] * 2, base + a.kc + cache_off[i] * 2, cbytes,
-                                 cudaMemcpyDeviceToHost, sg), "D2H k cache");
-          PP_TRY(cudaMemcpyAsync((char*)v_cache_host + cache_off[i] * 2, base + a.vc + cache_off[i] * 2, cbytes,
-                                 cudaMemcpyDeviceToHost, sg), "D2H v cache");
-        }
-        PP_TRY(cudaMemcpyAsync((char*)o_host + tok_off[i] * q_row, base + a.o + row * q_row, lengths[i] * q_row,
-                               cudaMemcpyDeviceToHost, sg), "D2H o");
-      }
+      gp.flags = pp::kFlagTablesReady;
+      PP_TRY(cudaMemcpyAsync(base + h.q_tok + tok0 * q_row, (const char*)q_host + tok0 * q_row, ntok * q_row,
+                             cudaMemcpyHostToDevice, sg), "H2D q");
+      PP_TRY(cudaMemcpyAsync(base + h.k_tok + tok0 * kv_row, (const char*)k_host + tok0 * kv_row, ntok * kv_row,
+                             cudaMemcpyHostToDevice, sg), "H2D k");
+      PP_TRY(cudaMemcpyAsync(base + h.v_tok + tok0 * kv_row, (const char*)v_host + tok0 * kv_row, ntok * kv_row,
+                             cudaMemcpyHostToDevice, sg), "H2D v");
+      mark(sg);
+      // padding rows of the packed buffers must be finite
+      PP_TRY(cudaMemsetAsync(base + h.q + rows0 * q_row, 0, nrows * q_row, sg), "memset packed q");
+      PP_TRY(cudaMemsetAsync(base + h.k + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed k");
+      PP_TRY(cudaMemsetAsync(base + h.v + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed v");
+      mark(sg);   // memsets
+      if ((st = pp::launch_tensorize(true, gq, base + h.q_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return st;
+      if ((st = pp::launch_tensorize(true, gk, base + h.k_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return st;
+      if ((st = pp::launch_tensorize(true, gv, base + h.v_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return st;
+      mark(sg);   // scatter
+      st = pp_prefill_attention(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), kg, gq, gk, gv, go,
+                                base + h.ws_attn + g * h.ws_attn_stride, static_cast<char*>(stage) + map_bytes, attn_tab,
+                                reinterpret_cast<int32_t*>(base + h.status), sg);
+      if (st != PP_OK) return st;
+      mark(sg);   // attention
+      st = pp_unpack_kv(&gp, G.bin_of.data(), G.off_of.data(), lengths + G.i0, kg, gk, gv, base + h.kc, base + h.vc,
+                        g_cache_off.data(), lengths + G.i0, base + h.ws_unpack + g * h.ws_unpack_stride,
+                        static_cast<char*>(stage) + map_bytes + attn_tab, unpack_tab, sg);
+      if (st != PP_OK) return st;
+      if ((st = pp::launch_tensorize(false, go, base + h.o_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return st;
+      mark(sg);
+      PP_TRY(cudaMemcpyAsync((char*)o_host + tok0 * q_row, base + h.o_tok + tok0 * q_row, ntok * q_row,
+                             cudaMemcpyDeviceToHost, sg), "D2H o");
+      PP_TRY(cudaMemcpyAsync((char*)k_cache_host + tok0 * kv_row, base + h.kc + tok0 * kv_row, ntok * kv_row,
+                             cudaMemcpyDeviceToHost, sg), "D2H k cache");
+      PP_TRY(cudaMemcpyAsync((char*)v_cache_host + tok0 * kv_row, base + h.vc + tok0 * kv_row, ntok * kv_row,
+                             cudaMemcpyDeviceToHost, sg), "D2H v cache");
+      mark(sg);
       PP_TRY(cudaEventRecord(pipe->done[g], sg), "event record");
       PP_TRY(cudaStreamWaitEvent(s, pipe->done[g], 0), "stream wait");
     }
     int32_t status = 0;
-    PP_TRY(cudaMemcpyAsync(&status, base + a.status, 4, cudaMemcpyDeviceToHost, s), "D2H status");
+    PP_TRY(cudaMemcpyAsync(&status, base + h.status, 4, cudaMemcpyDeviceToHost, s), "D2H status");
     PP_TRY(cudaStreamSynchronize(s), "stream synchronize");
+    if (trace) {
+      for (size_t i = 1; i < tev.size(); ++i) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, tev[0], tev[i]);
+        std::fprintf(stderr, "%s%.2f", (i - 1) % 6 == 0 ? "\n[pp_prefill_host] group: h2d, memset, scatter, attention, unpack+gather, d2h done (ms): " : ", ", ms);
+      }
+      std::fprintf(stderr, "\n");
+      for (cudaEvent_t ev : tev) cudaEventDestroy(ev);
+    }
 #undef PP_TRY
     return status == 0 ? PP_OK : PP_ERR_DEVICE_TIMEOUT;
   } catch (const std::bad_alloc&) {

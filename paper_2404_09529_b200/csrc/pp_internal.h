@@ -75,6 +75,11 @@ int launch_rope_table(const pp_attn_params& p, void* table, void* stream);
 int launch_unpack(const pp_attn_params& p, const int32_t* d_table, int32_t k, int64_t total_tokens,
                   const void* k_rot, const void* v, void* k_cache, void* v_cache, void* stream);
 
+// Row scatter (to_packed) / gather between a token-major tensor [T, row_bytes] and the packed layout.
+// d_map: device int64 tok_prefix[n_prompts + 1] followed by first_row[n_prompts].
+int launch_tensorize(bool to_packed, void* packed, void* tokens, const int64_t* d_map, int32_t n_prompts,
+                     int64_t total_tokens, int32_t row_bytes, void* stream);
+
 int launch_bounded_wait_selftest(int32_t* device_status, uint64_t limit_ns, void* stream);
 
 // Unpack table (int32 units): header 4 ints, then token_prefix[k+1], bin_of[k], off_of[k],

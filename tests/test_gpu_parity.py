@@ -162,15 +162,17 @@ def test_host_buffer_entry_point_matches_device_path():
     assert torch.equal(kc, ref.k_cache.cpu()) and torch.equal(vc, ref.v_cache.cpu())
 
 
-def test_host_buffer_entry_point_pipelined_groups():
-    """Large prompts make pp_prefill_host cut the bins into groups that it pipelines over its own
-    streams; the kernels of a group see fewer bins, so O may differ from the whole-batch run only
-    through the tile-to-CTA schedule (it does not: same tiles, same arithmetic) and the caches never."""
+@pytest.mark.parametrize("groups", [1, 3, 8])
+def test_host_buffer_entry_point_pipelined_groups(groups, monkeypatch):
+    """pp_prefill_host cuts large batches into groups of prompts, each packed on its own and run on
+    its own stream. Caches do not depend on the packing (bit-identical to the whole-batch run); O
+    depends on it only through the position of tile boundaries (summation order)."""
     import paper_2404_09529_b200 as pp
     lengths = np.array([900, 850, 700, 640, 512, 400, 333, 300, 128, 90, 60, 7], np.int32)
     hq, hkv, d, base = 8, 2, 128, 500000.0
     q, k, v = _random_case(lengths, hq, hkv, d, seed=5)
     ref = run_cuda(lengths, q, k, v, hq, hkv, d, base)
+    monkeypatch.setenv("PP_HOST_GROUPS", str(groups))
     params = pp.AttnParams(hq, hkv, d, base, 0.0, 0, 0, 0)
     nbytes = pp.pp_prefill_host_arena_bytes(params, lengths)
     arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
@@ -182,9 +184,13 @@ def test_host_buffer_entry_point_pipelined_groups():
         o.zero_(); kc.zero_(); vc.zero_()
         pp.pp_prefill_host(params, lengths, qh, kh, vh, o, kc, vc, arena, nbytes,
                            torch.cuda.current_stream().cuda_stream)
-        assert params.n_bins >= 4                      # several groups
+        assert params.capacity == 900 and params.n_bins >= 6
         assert torch.equal(kc, ref.k_cache.cpu()) and torch.equal(vc, ref.v_cache.cpu())
-        assert torch.equal(o, ref.o_tokens().cpu())
+        if groups == 1:
+            assert torch.equal(o, ref.o_tokens().cpu())
+        else:
+            diff = (o.float() - ref.o_tokens().cpu().float()).abs()
+            assert float(diff.max()) <= 2e-2 and float(diff.mean()) <= 5e-4
 
 
 def test_bounded_wait_gives_up_and_reports():
