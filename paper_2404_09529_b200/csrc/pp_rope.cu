@@ -160,6 +160,7 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
   __shared__ int32_t s_pos[kRuRows];              // restart position, -1 for padding rows
   __shared__ int64_t s_dst[kRuRows];              // cache element offset of (head 0, this position); -1: not cached
   __shared__ int64_t s_head_stride[kRuRows];      // cache_cap * D
+  __shared__ float4 s_tab[kRuRows][D / 4];          // (cos, sin) of j = 2g, 2g + 1 at each row's position
 
   const int64_t row0 = (int64_t)blockIdx.x * kRuRows;
   const int64_t n_rows = (int64_t)n_bins * capacity;
@@ -190,6 +191,12 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     s_head_stride[tid] = stride;
   }
   __syncthreads();
+  // each row's D/2 (cos, sin) pairs once, for all heads: D/4 16-byte loads per row, one per thread
+  for (int u = tid; u < kRuRows * (D / 4); u += kRopeThreads) {
+    const int r = u / (D / 4), g = u - r * (D / 4);
+    const int32_t pos = s_pos[r];
+    if (pos > 0) s_tab[r][g] = __ldg(reinterpret_cast<const float4*>(rope_table) + (size_t)g * (size_t)capacity + pos);
+  }
 
   // V rows first: plain 16-byte copies, four in flight per thread
   const int units_v = n_kv_heads * kVecs;
@@ -213,6 +220,7 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     for (int i = 0; i < kRuV; ++i)
       if (dsts[i] >= 0) *reinterpret_cast<uint4*>(v_cache + dsts[i]) = val[i];
   }
+  __syncthreads();
   // K rows: rotate, write back to the packed tensor and into the cache; two pairs in flight
   const int units_k = n_kv_heads * kPairUnits;
   for (int u0 = tid; u0 < kRuRows * units_k; u0 += kRuK * kRopeThreads) {
@@ -240,10 +248,9 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
       __nv_bfloat16* base = k + ((row0 + r) * n_kv_heads + head) * D;
       if (pos > 0) {
         float cs[8], sn[8];
-        const float4* tab = reinterpret_cast<const float4*>(rope_table) + pos;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const float4 t4 = __ldg(tab + (size_t)(c * 4 + q) * (size_t)capacity);
+          const float4 t4 = s_tab[r][c * 4 + q];
           cs[2 * q] = t4.x; sn[2 * q] = t4.y; cs[2 * q + 1] = t4.z; sn[2 * q + 1] = t4.w;
         }
         rotate8(lo[i], hi[i], cs, sn);
