@@ -1,0 +1,137 @@
+"""Two measurement sweeps over the prefill path, on synthetic batches (Sections 5.2 and 6 of the paper).
+
+``predictor``: batches of k prompts with lengths uniform in [1, 512]; for every batch the packed
+and the padded (full-batching) path are timed and the speedup is regressed on the two batch
+statistics the paper uses: the bin reduction r / k and the padding per prompt m - L / k
+(m = longest prompt, L = total tokens, r = bins after packing). Attention layer only.
+
+``dataset``: a stream of prompts is prefilled (a) prepacked as a whole and processed in launches
+of a fixed number of bins, (b) in batches of consecutive prompts after sorting the stream by
+length, each padded to its own maximum, (c) in batches in arrival order, padded. Reports useful
+tokens per second of each schedule.
+
+Both print one JSON object. They only marshal arguments: all arithmetic runs in the library.
+
+    python -m paper_2404_09529_b200.sweep predictor [--batches 40] [--k 16]
+    python -m paper_2404_09529_b200.sweep dataset [--prompts 4096] [--batch 16]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from .runner import PrefillBatch
+
+# Llama-2-7B attention layer shape
+HQ, HKV, D, BASE = 32, 32, 128, 10000.0
+
+
+def _time_ms(fn, iters: int = 5, warmup: int = 2) -> float:
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def _batch(lengths: np.ndarray, mode: str, gen: torch.Generator) -> PrefillBatch:
+    b = PrefillBatch(lengths, HQ, HKV, D, BASE, mode=mode)
+    t = int(lengths.sum())
+    q = torch.randn(t, HQ, D, generator=gen, device="cuda").to(torch.bfloat16)
+    k = torch.randn(t, HKV, D, generator=gen, device="cuda").to(torch.bfloat16)
+    v = torch.randn(t, HKV, D, generator=gen, device="cuda").to(torch.bfloat16)
+    b.load(q, k, v)
+    return b
+
+
+def predictor(n_batches: int, k: int, seed: int) -> dict:
+    rng = np.random.default_rng(seed)
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    rows = []
+    for _ in range(n_batches):
+        lengths = rng.integers(1, 513, size=k).astype(np.int32)
+        packed, padded = _batch(lengths, "packed", gen), _batch(lengths, "padded", gen)
+        ms_packed = _time_ms(lambda: packed.run_fused(repack=True))
+        ms_padded = _time_ms(lambda: padded.run_fused(repack=True))
+        assert packed.device_status() == 0 and padded.device_status() == 0
+        m, total, r = int(lengths.max()), int(lengths.sum()), int(packed.pack.n_bins)
+        rows.append({"r_over_k": r / k, "pad_per_prompt": m - total / k, "speedup": ms_padded / ms_packed,
+                     "ms_packed": ms_packed, "ms_padded": ms_padded})
+        del packed, padded
+    x = np.array([[1.0, row["r_over_k"], row["pad_per_prompt"]] for row in rows])
+    y = np.array([row["speedup"] for row in rows])
+    coef, *_ = np.linalg.lstsq(x, y, rcond=None)
+    pred = x @ coef
+    ss_res, ss_tot = float(((y - pred) ** 2).sum()), float(((y - y.mean()) ** 2).sum())
+    return {"sweep": "predictor", "k": k, "batches": n_batches, "lengths": "uniform int in [1, 512]",
+            "layer": {"n_q_heads": HQ, "n_kv_heads": HKV, "head_dim": D},
+            "speedup_mean": float(y.mean()), "speedup_min": float(y.min()), "speedup_max": float(y.max()),
+            "fit": {"intercept": float(coef[0]), "r_over_k": float(coef[1]), "pad_per_prompt": float(coef[2]),
+                    "r2": 1.0 - ss_res / ss_tot if ss_tot > 0 else 1.0},
+            "rows": rows}
+
+
+def dataset(n_prompts: int, batch: int, seed: int) -> dict:
+    rng = np.random.default_rng(seed)
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    lengths = np.clip(np.rint(np.exp(np.log(200.0) + 0.8 * rng.standard_normal(n_prompts))), 8, 2048).astype(np.int32)
+    total = int(lengths.sum())
+
+    def run_schedule(groups, mode):
+        ms = 0.0
+        for g in groups:
+            b = _batch(g, mode, gen)
+            ms += _time_ms(lambda: b.run_fused(repack=True), iters=3, warmup=1)
+            assert b.device_status() == 0
+            del b
+        return ms
+
+    # (a) prepack the whole stream, launches of `batch` prompts' worth of tokens each: the packer is
+    # run per launch group of consecutive prompts large enough to fill many bins
+    per_launch = batch * 16
+    packed_groups = [lengths[i:i + per_launch] for i in range(0, n_prompts, per_launch)]
+    ms_prepacked = run_schedule(packed_groups, "packed")
+    # (b) length-ordered batching: sort, then padded batches of `batch`
+    order = np.sort(lengths)
+    ms_sorted = run_schedule([order[i:i + batch] for i in range(0, n_prompts, batch)], "padded")
+    # (c) arrival order, padded batches of `batch`
+    ms_arrival = run_schedule([lengths[i:i + batch] for i in range(0, n_prompts, batch)], "padded")
+    tps = lambda ms: total / (ms * 1e-3)
+    return {"sweep": "dataset", "prompts": n_prompts, "total_tokens": total,
+            "lengths": "lognormal(median 200, sigma 0.8) clipped to [8, 2048]",
+            "layer": {"n_q_heads": HQ, "n_kv_heads": HKV, "head_dim": D},
+            "prepacked": {"prompts_per_launch": per_launch, "ms": ms_prepacked, "tokens_per_s": tps(ms_prepacked)},
+            "length_ordered_padded": {"batch": batch, "ms": ms_sorted, "tokens_per_s": tps(ms_sorted)},
+            "arrival_order_padded": {"batch": batch, "ms": ms_arrival, "tokens_per_s": tps(ms_arrival)},
+            "speedup_vs_arrival_order": ms_arrival / ms_prepacked,
+            "speedup_vs_length_ordered": ms_sorted / ms_prepacked}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    sub = ap.add_subparsers(dest="cmd", required=True)
+    p = sub.add_parser("predictor")
+    p.add_argument("--batches", type=int, default=40)
+    p.add_argument("--k", type=int, default=16)
+    p.add_argument("--seed", type=int, default=0)
+    d = sub.add_parser("dataset")
+    d.add_argument("--prompts", type=int, default=4096)
+    d.add_argument("--batch", type=int, default=16)
+    d.add_argument("--seed", type=int, default=0)
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("the sweeps need a GPU: the library has no CPU path")
+    out = predictor(args.batches, args.k, args.seed) if args.cmd == "predictor" else dataset(args.prompts, args.batch, args.seed)
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

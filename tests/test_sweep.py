@@ -1,0 +1,24 @@
+"""The two measurement sweeps run end to end on small inputs (GPU only: the library has no CPU path)."""
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+def test_predictor_sweep_small():
+    from paper_2404_09529_b200 import sweep
+    out = sweep.predictor(n_batches=4, k=8, seed=1)
+    assert out["batches"] == 4 and len(out["rows"]) == 4
+    for row in out["rows"]:
+        assert 0.0 < row["r_over_k"] <= 1.0 and row["pad_per_prompt"] >= 0.0
+        assert row["ms_packed"] > 0.0 and row["ms_padded"] > 0.0
+    assert set(out["fit"]) == {"intercept", "r_over_k", "pad_per_prompt", "r2"}
+
+
+def test_dataset_sweep_small():
+    from paper_2404_09529_b200 import sweep
+    out = sweep.dataset(n_prompts=64, batch=8, seed=1)
+    assert out["total_tokens"] > 0
+    for key in ("prepacked", "length_ordered_padded", "arrival_order_padded"):
+        assert out[key]["tokens_per_s"] > 0.0
+    # with a lognormal length mix, padding to the batch maximum in arrival order wastes the most
+    assert out["speedup_vs_arrival_order"] > 1.0
