@@ -1,14 +1,14 @@
 /*
  * prepack-b200: C ABI of the prepacked-prefill attention hot path for NVIDIA B200 (sm_100a).
  *
- * The library follows Algorithm 1 ("Prepacking") of arXiv 2404.09529:
- *   line 4   BINPACK            -> pp_pack                 (host)
- *   line 5   TENSORIZE          -> layout contract below   (no call)
- *   line 6   INDEPENDENT-MASK   -> applied inside pp_prefill_attention, never materialised
- *   line 7   RESTART-PE         -> applied inside pp_prefill_attention (rotary), also
- *                                  available as explicit ids from pp_fill_position_ids
- *   line 8   forward + UNPACK   -> pp_prefill_attention (the attention of one layer) and
- *                                  pp_unpack_kv
+ * The library follows the steps of Algorithm 1 ("Prepacking") of arXiv 2404.09529:
+ *   BINPACK            -> pp_pack                 (host)
+ *   TENSORIZE          -> layout contract below   (no call)
+ *   INDEPENDENT-MASK   -> applied inside pp_prefill_attention, never materialised
+ *   RESTART-PE         -> applied inside pp_prefill_attention (rotary), also
+ *                         available as explicit ids from pp_fill_position_ids
+ *   forward + UNPACK   -> pp_prefill_attention (the attention of one layer) and
+ *                         pp_unpack_kv
  *
  * Conventions
  *   - Every function returns an int status (PP_OK = 0, errors < 0). Nothing aborts or throws.
@@ -58,7 +58,7 @@ typedef struct pp_attn_params {
   int32_t head_dim;      /* D: 64 or 128                                                       */
   float rope_base;       /* rotary base; theta_j = base^(-2j/D), pairs (j, j + D/2)             */
   float softmax_scale;   /* 0 selects 1/sqrt(D) (Section 2.1)                                  */
-  int32_t capacity;      /* M: rows per bin (Algorithm 1 line 3: the longest prompt)           */
+  int32_t capacity;      /* M: rows per bin (Algorithm 1 (bin size): the longest prompt)           */
   int32_t n_bins;        /* R                                                                  */
   int32_t flags;         /* PP_FLAG_* or 0                                                     */
 } pp_attn_params;
@@ -71,7 +71,7 @@ const char* pp_strerror(int status);
 const char* pp_last_cuda_error(void);
 
 /*
- * BINPACK -- Section 3.1 and Algorithm 1 lines 2-4. Host only, deterministic.
+ * BINPACK -- Section 3.1 and Algorithm 1 (bin size, BINPACK). Host only, deterministic.
  * First-fit-decreasing of k prompt lengths into bins of `capacity` rows (0 selects the longest
  * prompt, the paper's choice). Items are taken by length descending, equal lengths by original
  * index ascending; each goes to the lowest-numbered bin with room, else opens a new bin; bins
@@ -93,7 +93,7 @@ int pp_pack(const int32_t* lengths, int32_t k, int32_t capacity,
             int32_t* bin_of, int32_t* off_of);
 
 /*
- * RESTART-PE as explicit ids -- Section 3.2, Algorithm 1 line 7. Host only.
+ * RESTART-PE as explicit ids -- Section 3.2, Algorithm 1 (RESTART-PE). Host only.
  * position_ids [n_bins*capacity]: 0,1,2,... restarting at every segment start; padding rows 0.
  * segment_ids  [n_bins*capacity]: index into the seg_* arrays; padding rows -1. Either output
  * may be NULL. Errors: PP_ERR_INVALID_ARG on NULL inputs or segments that do not tile a bin
@@ -110,7 +110,7 @@ int pp_fill_position_ids(int32_t n_bins, int32_t capacity, const int32_t* bin_se
 size_t pp_prefill_workspace_bytes(const pp_attn_params* params, int32_t k);
 
 /*
- * Prefill attention over the packed batch -- Algorithm 1 lines 6-8 for one attention layer:
+ * Prefill attention over the packed batch -- Algorithm 1 (INDEPENDENT-MASK to UNPACK) for one attention layer:
  * restart rotary encoding of q and k (Section 3.2), then per bin and query head
  *   o_i = sum_j softmax_j(q'_i . k'_j * scale) v_j   over keys j of the SAME prompt with j <= i
  * (independent mask M' of Section 3.2: a lower-triangular block per prompt span, zero elsewhere).
@@ -143,7 +143,7 @@ int pp_prefill_attention(const pp_attn_params* params,
                          int32_t* device_status, void* stream);
 
 /*
- * The same result as pp_prefill_attention followed by pp_unpack_kv (Algorithm 1 lines 6-8 for one
+ * The same result as pp_prefill_attention followed by pp_unpack_kv (Algorithm 1 (INDEPENDENT-MASK to UNPACK) for one
  * attention layer), with fewer passes over HBM: one kernel rotates K, writes it back to the packed
  * tensor and into the per-prompt K caches and copies V into the V caches; the attention kernel
  * rotates each Q tile on the fly, so q is read only.
@@ -183,7 +183,7 @@ int pp_selftest_bounded_wait(int32_t* device_status, uint32_t limit_ms, void* st
 size_t pp_unpack_workspace_bytes(int32_t k);
 
 /*
- * UNPACK -- Algorithm 1 line 8, Section 4.3: copy each prompt's rotated keys and its values out
+ * UNPACK -- Algorithm 1 (UNPACK), Section 4.3: copy each prompt's rotated keys and its values out
  * of the packed tensors into that prompt's own cache, in original prompt order.
  *   cache[i][h][p][:] = packed[bin_of[i], off_of[i] + p, h, :]   for p < lengths[i]
  *   bin_of, off_of, lengths  host [k], original prompt order (lengths may be shorter than the
@@ -225,7 +225,7 @@ int pp_unpack_kv_static(const pp_attn_params* params,
                         const int64_t* cache_off, const int32_t* cache_cap, void* stream);
 
 /*
- * Whole path from host memory (Algorithm 1 lines 2-8 for one attention layer), for callers whose
+ * Whole path from host memory (Algorithm 1 (bin size to UNPACK) for one attention layer), for callers whose
  * tensors live on the host. Every tensor goes up in large contiguous copies, is laid out as the
  * packed batch by a device kernel (TENSORIZE, padding rows zeroed), pp_prefill_attention and
  * pp_unpack_kv run there, O is gathered back into token order and the outputs are copied back;

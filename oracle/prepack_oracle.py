@@ -18,10 +18,10 @@ What is computed, and where the paper fixes it:
   and query head h reads KV head h // (Hq // Hkv); the positional encoding is
   rotary in the "rotate-half" pairing (j, j + D/2) with theta_j = base^(-2j/D);
   the cache of one layer is K after the rotation and V unrotated.
-* ``ffd_pack`` is textbook first-fit-decreasing (Section 3.1, Algorithm 1 line 4)
+* ``ffd_pack`` is textbook first-fit-decreasing (Section 3.1, Algorithm 1 (BINPACK))
   with the tie rules spelled out in its docstring.
 * ``restart_position_ids`` / ``independent_mask`` / ``packed_dense_prefill`` spell
-  out Algorithm 1 lines 5-8 on dense tensors (TENSORIZE, INDEPENDENT-MASK,
+  out Algorithm 1 (TENSORIZE to UNPACK) on dense tensors (TENSORIZE, INDEPENDENT-MASK,
   RESTART-PE, UNPACK); ``padded_prefill`` is the full-batching baseline of
   Section 4.2. They exist so that tests can check the paper's exactness claim
   against ``prefill_prompt``.
@@ -156,7 +156,7 @@ def brute_force_prompt(q, k, v, base: float):
 
 
 # --------------------------------------------------------------------------- #
-# BINPACK: first-fit-decreasing (Section 3.1; Algorithm 1 line 4)
+# BINPACK: first-fit-decreasing (Section 3.1; Algorithm 1 (BINPACK))
 # --------------------------------------------------------------------------- #
 
 
@@ -167,7 +167,7 @@ def ffd_pack(lengths, capacity: int = 0):
     descending, equal lengths by original index ascending; each item goes into the
     lowest-numbered open bin with enough room left, else a new bin is opened; bins
     are numbered in creation order and hold their items in placement order.
-    capacity == 0 means the longest prompt (Algorithm 1 line 3).
+    capacity == 0 means the longest prompt (Algorithm 1 (bin size)).
 
     Returns a dict of int lists:
       n_bins, capacity,
@@ -218,7 +218,7 @@ def ffd_pack(lengths, capacity: int = 0):
 
 
 # --------------------------------------------------------------------------- #
-# Algorithm 1 lines 5-8 on dense tensors (cross-check formulations)
+# Algorithm 1 (TENSORIZE to UNPACK) on dense tensors (cross-check formulations)
 # --------------------------------------------------------------------------- #
 
 

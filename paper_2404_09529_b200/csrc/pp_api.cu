@@ -1,5 +1,5 @@
 // C-ABI entry points that touch the device: argument validation, table upload, kernel launches.
-// Algorithm 1 lines 5-8 of the prepacking paper; see include/pp.h for the contracts.
+// Algorithm 1 (TENSORIZE to UNPACK) of the prepacking paper; see include/pp.h for the contracts.
 #include <cuda_runtime.h>
 
 #include <algorithm>

@@ -1,6 +1,6 @@
 // Host side of the prepack-b200 library: BINPACK (first-fit-decreasing), RESTART-PE ids,
 // status strings, and the tile work list that the attention kernel walks.
-// Algorithm 1 lines 2-7 and Sections 3.1-3.2 of the prepacking paper.
+// Algorithm 1 (bin size to RESTART-PE) and Sections 3.1-3.2 of the prepacking paper.
 #include "pp_internal.h"
 
 #include <algorithm>

@@ -1,4 +1,4 @@
-// Restart rotary positional encoding over the packed batch (Section 3.2, Algorithm 1 line 7).
+// Restart rotary positional encoding over the packed batch (Section 3.2, Algorithm 1 (RESTART-PE)).
 // Each row's position is its bin-local row index minus the start row of the prompt it belongs
 // to; Q and K rows are rotated in place. HBM-bound: every element is read once and written once.
 #include <cuda_bf16.h>
@@ -137,7 +137,7 @@ rope_table_kernel(float2* __restrict__ table, int32_t capacity, int32_t half,
   table[((size_t)(j >> 1) * capacity + pos) * 2 + (j & 1)] = make_float2(cs, sn);
 }
 
-// Fused K rotation + UNPACK (Algorithm 1 lines 7-8 in one pass over K and V): every real packed
+// Fused K rotation + UNPACK (Algorithm 1 (RESTART-PE to UNPACK) in one pass over K and V): every real packed
 // row of K is rotated (cos/sin from the table), written back to the packed tensor (the attention
 // kernel reads it there) and into its prompt's K cache; the V row is copied into the V cache.
 struct SegExt {                    // per-segment arrays appended to the prefill table

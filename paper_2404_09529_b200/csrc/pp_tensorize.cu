@@ -1,4 +1,4 @@
-// TENSORIZE (Algorithm 1 line 5) on the device, for the host-buffer entry point: rows of a
+// TENSORIZE (Algorithm 1 (TENSORIZE)) on the device, for the host-buffer entry point: rows of a
 // token-major tensor [T, H, D] (prompts back to back in original order) are scattered into the packed
 // [R, M, H, D] layout, or gathered back from it. A row is H * D contiguous elements on both sides, so
 // this is a row permutation by 16-byte copies; it lets the host side move each tensor with one large

@@ -1,4 +1,4 @@
-// UNPACK (Algorithm 1 line 8, Section 4.3): scatter every prompt's rotated keys and its values
+// UNPACK (Algorithm 1 (UNPACK), Section 4.3): scatter every prompt's rotated keys and its values
 // from the packed [R, M, Hkv, D] tensors into that prompt's own [Hkv, cap, D] cache, in
 // original prompt order. Pure 16-byte copies; HBM-bound.
 #include <cuda_bf16.h>

@@ -30,7 +30,7 @@ def _bins_of(pack):
 
 
 def test_pack_tiny_hand_worked():
-    """Algorithm 1 line 4 on the tiny workload, against the hand-worked fixture."""
+    """Algorithm 1 (BINPACK) on the tiny workload, against the hand-worked fixture."""
     g = json.load(open(os.path.join(GOLDEN, "pack_tiny.json")))
     pack = orc.ffd_pack(g["lengths"], 0)
     bins, starts = _bins_of(pack)
