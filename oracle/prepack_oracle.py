@@ -26,11 +26,14 @@ What is computed, and where the paper fixes it:
   Section 4.2. They exist so that tests can check the paper's exactness claim
   against ``prefill_prompt``.
 * ``brute_force_prompt`` is a pure-Python loop version for tiny inputs.
+* ``decode_step`` is one generation step over a prompt's own caches (Section 7,
+  prepacking for generation): the new token at position l, appended and attended.
 
 Parity pins (tests/test_oracle_pins.py): complex-number form of the rotation,
 torch SDPA in float64, closed forms (identical keys, identical values, first
 row), packed == padded == alone, zero cross-prompt probability mass, brute force,
-and the hand-worked packing of the tiny workload. No function is unpinned.
+the hand-worked packing of the tiny workload, and decode step == last row of the
+extended prompt's prefill. No function is unpinned.
 
 All floating point here is float64. Inputs are expected to be bf16-representable
 values already upcast to float64 by the caller.
@@ -326,3 +329,38 @@ def padded_prefill(qs, ks, vs, base: float):
         kcs.append(np.transpose(k_rot[:l], (1, 0, 2)))
         vcs.append(np.transpose(pad(v)[:l], (1, 0, 2)))
     return os_, kcs, vcs
+
+
+# --------------------------------------------------------------------------- #
+# One generation step over per-prompt caches (Section 7: prepacking for generation)
+# --------------------------------------------------------------------------- #
+
+
+def decode_step(q_new, k_new, v_new, k_cache, v_cache, base: float):
+    """The token that follows a prompt of l tokens, for one prompt alone.
+
+    q_new [Hq, D], k_new, v_new [Hkv, D]: the new token's (unrotated) projections; k_cache
+    [Hkv, l, D] holds the rotated keys of positions 0..l-1 and v_cache [Hkv, l, D] the values.
+    The new token sits at position l: its query and key are rotated by l * theta_j, key and value
+    are appended to the caches, and the query attends to all l + 1 positions (the causal mask of
+    the last row of an (l + 1)-token prompt). Returns (o [Hq, D], k_cache' [Hkv, l+1, D],
+    v_cache' [Hkv, l+1, D]). Everything float64.
+    """
+    q_new, k_new, v_new = (np.asarray(x, dtype=np.float64) for x in (q_new, k_new, v_new))
+    k_cache, v_cache = np.asarray(k_cache, dtype=np.float64), np.asarray(v_cache, dtype=np.float64)
+    hq, d = q_new.shape
+    hkv, l, _ = k_cache.shape
+    g = hq // hkv
+    pos = np.array([l], dtype=np.int64)
+    q_rot = rope_rotate(q_new[None], pos, base)[0]             # [Hq, D]
+    k_rot = rope_rotate(k_new[None], pos, base)[0]             # [Hkv, D]
+    k_all = np.concatenate([k_cache, k_rot[:, None, :]], axis=1)
+    v_all = np.concatenate([v_cache, v_new[:, None, :]], axis=1)
+    o = np.empty((hq, d), dtype=np.float64)
+    scale = 1.0 / math.sqrt(d)
+    for h in range(hq):
+        s = (k_all[h // g] @ q_rot[h]) * scale                 # [l + 1]
+        p = np.exp(s - s.max())
+        p /= p.sum()
+        o[h] = p @ v_all[h // g]
+    return o, k_all, v_all

@@ -297,3 +297,35 @@ def test_restart_positions_matter_for_k_cache():
                        atol=1e-13)
     wrong = np.transpose(orc.rope_rotate(ks[1], np.arange(6, 10), 10000.0), (1, 0, 2))
     assert np.max(np.abs(kc[1] - wrong)) > 1e-3
+
+
+def test_decode_step_equals_last_row_of_the_extended_prompt():
+    """Pin of the generation step: decoding token l from the caches of tokens 0..l-1 must give the
+    last attention row and the caches of an (l + 1)-token prefill (Sections 3.2 and 7)."""
+    rng = np.random.default_rng(11)
+    for (l, hq, hkv, d) in [(1, 2, 2, 8), (5, 4, 2, 16), (37, 4, 1, 64)]:
+        q = rng.standard_normal((l + 1, hq, d))
+        k = rng.standard_normal((l + 1, hkv, d))
+        v = rng.standard_normal((l + 1, hkv, d))
+        o_full, kc_full, vc_full = orc.prefill_prompt(q, k, v, 10000.0)
+        _, kc, vc = orc.prefill_prompt(q[:l], k[:l], v[:l], 10000.0)
+        o, kc2, vc2 = orc.decode_step(q[l], k[l], v[l], kc, vc, 10000.0)
+        assert np.max(np.abs(o - o_full[l])) < 1e-12
+        assert np.max(np.abs(kc2 - kc_full)) < 1e-12 and np.array_equal(vc2, vc_full)
+
+
+def test_decode_step_closed_forms():
+    """All cached values equal to the new value: the output is that value whatever the scores; an
+    empty history cannot exist (l >= 1), but l = 1 with identical keys gives the mean of two values."""
+    rng = np.random.default_rng(12)
+    hq, hkv, d, l = 4, 2, 16, 9
+    row = rng.standard_normal((hkv, d))
+    kc = rng.standard_normal((hkv, l, d))
+    vc = np.repeat(row[:, None, :], l, axis=1)
+    o, _, _ = orc.decode_step(rng.standard_normal((hq, d)), rng.standard_normal((hkv, d)), row, kc, vc, 5e5)
+    assert np.max(np.abs(o - np.repeat(row, hq // hkv, axis=0))) < 1e-12
+    # a zero query gives uniform weights over the l + 1 positions
+    vc = rng.standard_normal((hkv, l, d))
+    v_new = rng.standard_normal((hkv, d))
+    o, _, v_all = orc.decode_step(np.zeros((hq, d)), rng.standard_normal((hkv, d)), v_new, kc, vc, 5e5)
+    assert np.max(np.abs(o - np.repeat(v_all.mean(axis=1), hq // hkv, axis=0))) < 1e-12
