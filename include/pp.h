@@ -225,6 +225,32 @@ int pp_unpack_kv_static(const pp_attn_params* params,
                         const int64_t* cache_off, const int32_t* cache_cap, void* stream);
 
 /*
+ * One generation step over the per-prompt caches -- Section 7 (prepacking for generation). For
+ * every prompt i the new token sits at position lengths[i] (the number of tokens its caches hold):
+ * its query and key are rotated by that position, the rotated key and the value are appended to
+ * the caches at row lengths[i], and the query attends to rows 0 .. lengths[i]. The caches are the
+ * unpadded per-prompt blocks that pp_unpack_kv / pp_prefill_fused fill, so the step reads exactly
+ * the keys and values each prompt has, whatever the other prompts' lengths are.
+ *   params       n_q_heads, n_kv_heads (at most 8 query heads per KV head), head_dim, rope_base,
+ *                softmax_scale are read; capacity, n_bins and flags are ignored
+ *   lengths      host [k]: tokens already in each prompt's caches (>= 1)
+ *   q_new        device [k, Hq, D] bf16, k_new / v_new device [k, Hkv, D] bf16: the new tokens' raw
+ *                projections, read only
+ *   o            device [k, Hq, D] bf16 out
+ *   k_cache, v_cache, cache_off, cache_cap   as in pp_unpack_kv; cache_cap[i] > lengths[i]
+ *   workspace    device, >= pp_decode_workspace_bytes(params, lengths, k), 256-byte aligned;
+ *                host_workspace: host staging of the same size or at least the table part (pinned
+ *                memory keeps the call asynchronous)
+ * Asynchronous on `stream`. Errors: PP_ERR_INVALID_ARG, PP_ERR_LENGTH (no room for one more token),
+ * PP_ERR_UNSUPPORTED (head_dim, group size), PP_ERR_ALIGNMENT, PP_ERR_BUFFER_TOO_SMALL, PP_ERR_CUDA.
+ */
+size_t pp_decode_workspace_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k);
+int pp_decode_step(const pp_attn_params* params, const int32_t* lengths, int32_t k,
+                   const void* q_new, const void* k_new, const void* v_new, void* o,
+                   void* k_cache, void* v_cache, const int64_t* cache_off, const int32_t* cache_cap,
+                   void* workspace, void* host_workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Whole path from host memory (Algorithm 1 (bin size to UNPACK) for one attention layer), for callers whose
  * tensors live on the host. Every tensor goes up in large contiguous copies, is laid out as the
  * packed batch by a device kernel (TENSORIZE, padding rows zeroed), pp_prefill_attention and

@@ -5,7 +5,8 @@ the path (packing, restart rotary encoding, packed attention, KV unpack) runs in
 library. PyTorch is used by callers only for device memory and streams.
 """
 from .binding import (PP_FLAG_ROPE_ONLY, PP_FLAG_SKIP_ROPE, AttnParams, Packing, PrepackError,
-                      Workspaces, lib_path, load_library, pp_fill_position_ids,
+                      Workspaces, lib_path, load_library, pp_decode_step, pp_decode_workspace_bytes,
+                      pp_fill_position_ids,
                       pp_last_cuda_error, pp_pack, pp_prefill_attention, pp_prefill_fused,
                       pp_prefill_fused_workspace_bytes, pp_prefill_host,
                       pp_prefill_host_arena_bytes, pp_prefill_workspace_bytes, pp_selftest_bounded_wait, pp_strerror,
@@ -14,7 +15,7 @@ from .binding import (PP_FLAG_ROPE_ONLY, PP_FLAG_SKIP_ROPE, AttnParams, Packing,
 
 __all__ = [
     "PP_FLAG_ROPE_ONLY", "PP_FLAG_SKIP_ROPE", "AttnParams", "Packing", "PrepackError", "Workspaces",
-    "lib_path", "load_library", "pp_fill_position_ids", "pp_last_cuda_error", "pp_pack",
+    "lib_path", "load_library", "pp_decode_step", "pp_decode_workspace_bytes", "pp_fill_position_ids", "pp_last_cuda_error", "pp_pack",
     "pp_prefill_attention", "pp_prefill_fused", "pp_prefill_fused_workspace_bytes", "pp_prefill_host", "pp_prefill_host_arena_bytes",
     "pp_prefill_workspace_bytes", "pp_selftest_bounded_wait", "pp_strerror", "pp_unpack_kv", "pp_unpack_kv_static",
     "pp_unpack_static_max_prompts", "pp_unpack_workspace_bytes",

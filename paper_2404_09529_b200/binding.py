@@ -66,6 +66,9 @@ def load_library():
                                         ctypes.c_size_t, vp]),
         "pp_unpack_static_max_prompts": (ctypes.c_int32, []),
         "pp_unpack_kv_static": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, i64p, i32p, vp]),
+        "pp_decode_workspace_bytes": (ctypes.c_size_t, [pp, i32p, ctypes.c_int32]),
+        "pp_decode_step": (ctypes.c_int, [pp, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp, i64p, i32p, vp, vp,
+                                          ctypes.c_size_t, vp]),
         "pp_prefill_host_arena_bytes": (ctypes.c_size_t, [pp, i32p, ctypes.c_int32]),
         "pp_prefill_host": (ctypes.c_int, [pp, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]),
     }
@@ -173,6 +176,22 @@ def pp_prefill_fused(params: AttnParams, pack: Packing, lengths, q, k, v, o, k_c
         _addr(v_cache), co.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), _p32(cc), _addr(workspace),
         _addr(host_workspace), workspace_bytes, _addr(device_status), stream)
     _check(st, "pp_prefill_fused")
+
+
+def pp_decode_workspace_bytes(params: AttnParams, lengths) -> int:
+    l = _i32(lengths)
+    return int(load_library().pp_decode_workspace_bytes(ctypes.byref(params), _p32(l), int(l.shape[0])))
+
+
+def pp_decode_step(params: AttnParams, lengths, q_new, k_new, v_new, o, k_cache, v_cache, cache_off, cache_cap,
+                   workspace, host_workspace, workspace_bytes: int, stream: int = 0) -> None:
+    l, cc = _i32(lengths), _i32(cache_cap)
+    co = np.ascontiguousarray(np.asarray(cache_off, dtype=np.int64))
+    st = load_library().pp_decode_step(
+        ctypes.byref(params), _p32(l), int(l.shape[0]), _addr(q_new), _addr(k_new), _addr(v_new), _addr(o),
+        _addr(k_cache), _addr(v_cache), co.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), _p32(cc),
+        _addr(workspace), _addr(host_workspace), workspace_bytes, stream)
+    _check(st, "pp_decode_step")
 
 
 def pp_selftest_bounded_wait(device_status, limit_ms: int, stream: int = 0) -> None:

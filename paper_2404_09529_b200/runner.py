@@ -131,3 +131,63 @@ class PrefillBatch:
         off = int(self.cache_off[i])
         shape = (self.hkv, int(self.cache_cap[i]), self.d)
         return self.k_cache[off:off + n].view(shape), self.v_cache[off:off + n].view(shape)
+
+
+class DecodeBatch:
+    """Per-prompt KV caches with room to grow, and one generation step at a time through
+    pp_decode_step. Memory plumbing only: `adopt` copies the caches a PrefillBatch has filled into
+    blocks of capacity lengths[i] + room."""
+
+    def __init__(self, lengths, n_q_heads: int, n_kv_heads: int, head_dim: int, rope_base: float,
+                 room: int = 32, device: str = "cuda", softmax_scale: float = 0.0):
+        self.device = torch.device(device)
+        self.lengths = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32)).copy()
+        self.k = int(self.lengths.shape[0])
+        self.hq, self.hkv, self.d = n_q_heads, n_kv_heads, head_dim
+        self.cache_cap = (self.lengths + room).astype(np.int32)
+        prefix = np.concatenate([[0], np.cumsum(self.cache_cap.astype(np.int64))])
+        self.cache_off = (prefix[:-1] * n_kv_heads * head_dim).astype(np.int64)
+        pool = int(prefix[-1]) * n_kv_heads * head_dim
+        self.k_cache = torch.zeros(pool, dtype=torch.bfloat16, device=self.device)
+        self.v_cache = torch.zeros(pool, dtype=torch.bfloat16, device=self.device)
+        self.params = B.AttnParams(n_q_heads, n_kv_heads, head_dim, rope_base, softmax_scale, 1, 1, 0)
+        self.o = torch.zeros((self.k, n_q_heads, head_dim), dtype=torch.bfloat16, device=self.device)
+        self._ws_bytes = 0
+        self._ws = self._host = None
+
+    def caches(self, i: int):
+        """(k_cache_i, v_cache_i) as [Hkv, cap_i, D] views; rows [0, lengths[i]) are filled."""
+        cap = int(self.cache_cap[i])
+        n = cap * self.hkv * self.d
+        off = int(self.cache_off[i])
+        shape = (self.hkv, cap, self.d)
+        return self.k_cache[off:off + n].view(shape), self.v_cache[off:off + n].view(shape)
+
+    def adopt(self, prefill: PrefillBatch) -> None:
+        for i in range(self.k):
+            src_k, src_v = prefill.caches(i)
+            dst_k, dst_v = self.caches(i)
+            l = int(self.lengths[i])
+            dst_k[:, :l].copy_(src_k[:, :l])
+            dst_v[:, :l].copy_(src_v[:, :l])
+
+    def step(self, q_new: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor) -> torch.Tensor:
+        """One token per prompt: q_new [k, Hq, D], k_new / v_new [k, Hkv, D] bf16 on the device."""
+        need = B.pp_decode_workspace_bytes(self.params, self.lengths)
+        if need > self._ws_bytes:
+            self._ws_bytes = need + (need >> 2)        # lengths grow by one per step
+            self._ws = torch.empty(self._ws_bytes, dtype=torch.uint8, device=self.device)
+            self._host = [torch.empty(self._ws_bytes, dtype=torch.uint8).pin_memory() for _ in range(2)]
+            self._copied = [None, None]                # event after the upload that last read each staging buffer
+            self._turn = 0
+        slot = self._turn & 1
+        self._turn += 1
+        if self._copied[slot] is not None:
+            self._copied[slot].synchronize()
+        B.pp_decode_step(self.params, self.lengths, q_new, k_new, v_new, self.o, self.k_cache, self.v_cache,
+                         self.cache_off, self.cache_cap, self._ws, self._host[slot], self._ws_bytes,
+                         torch.cuda.current_stream().cuda_stream)
+        self._copied[slot] = torch.cuda.Event()
+        self._copied[slot].record()
+        self.lengths += 1
+        return self.o

@@ -10,10 +10,15 @@ of a fixed number of bins, (b) in batches of consecutive prompts after sorting t
 length, each padded to its own maximum, (c) in batches in arrival order, padded. Reports useful
 tokens per second of each schedule.
 
-Both print one JSON object. They only marshal arguments: all arithmetic runs in the library.
+``generation``: decode steps over the per-prompt caches (Section 7: a batch of nine prompts of one
+token and one of 1000 tokens, 20 generated tokens), against the same steps with every prompt
+declared as long as the longest (what padded caches cost).
+
+Each prints one JSON object. They only marshal arguments: all arithmetic runs in the library.
 
     python -m paper_2404_09529_b200.sweep predictor [--batches 40] [--k 16]
     python -m paper_2404_09529_b200.sweep dataset [--prompts 4096] [--batch 16]
+    python -m paper_2404_09529_b200.sweep generation [--tokens 20]
 """
 from __future__ import annotations
 
@@ -23,7 +28,7 @@ import json
 import numpy as np
 import torch
 
-from .runner import PrefillBatch
+from .runner import DecodeBatch, PrefillBatch
 
 # Llama-2-7B attention layer shape
 HQ, HKV, D, BASE = 32, 32, 128, 10000.0
@@ -115,6 +120,40 @@ def dataset(n_prompts: int, batch: int, seed: int) -> dict:
             "speedup_vs_length_ordered": ms_sorted / ms_prepacked}
 
 
+def generation(n_tokens: int, seed: int) -> dict:
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+
+    def per_token_ms(lengths):
+        dec = DecodeBatch(lengths, HQ, HKV, D, BASE, room=n_tokens + 4)
+        dec.k_cache.normal_(generator=gen)              # any finite cache contents cost the same
+        dec.v_cache.normal_(generator=gen)
+        k = len(lengths)
+        qn = torch.randn(k, HQ, D, generator=gen, device="cuda").to(torch.bfloat16)
+        kn = torch.randn(k, HKV, D, generator=gen, device="cuda").to(torch.bfloat16)
+        vn = torch.randn(k, HKV, D, generator=gen, device="cuda").to(torch.bfloat16)
+        dec.step(qn, kn, vn)                             # warm-up (also sizes the workspace)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_tokens):
+            dec.step(qn, kn, vn)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n_tokens
+
+    cases = {"toy_9x1_1x1000": np.array([1] * 9 + [1000], np.int32),
+             "lognormal_64": np.clip(np.rint(np.exp(np.log(200.0) + 0.8 * np.random.default_rng(seed).standard_normal(64))),
+                                     8, 2048).astype(np.int32)}
+    out = {"sweep": "generation", "tokens": n_tokens, "layer": {"n_q_heads": HQ, "n_kv_heads": HKV, "head_dim": D}}
+    for name, lengths in cases.items():
+        ms_true = per_token_ms(lengths)
+        ms_padded = per_token_ms(np.full_like(lengths, lengths.max()))
+        out[name] = {"prompts": int(len(lengths)), "cached_tokens": int(lengths.sum()),
+                     "padded_cached_tokens": int(lengths.max()) * int(len(lengths)),
+                     "ms_per_token": ms_true, "ms_per_token_padded": ms_padded, "speedup": ms_padded / ms_true}
+    return out
+
+
 def main() -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -126,10 +165,18 @@ def main() -> None:
     d.add_argument("--prompts", type=int, default=4096)
     d.add_argument("--batch", type=int, default=16)
     d.add_argument("--seed", type=int, default=0)
+    gsub = sub.add_parser("generation")
+    gsub.add_argument("--tokens", type=int, default=20)
+    gsub.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("the sweeps need a GPU: the library has no CPU path")
-    out = predictor(args.batches, args.k, args.seed) if args.cmd == "predictor" else dataset(args.prompts, args.batch, args.seed)
+    if args.cmd == "predictor":
+        out = predictor(args.batches, args.k, args.seed)
+    elif args.cmd == "dataset":
+        out = dataset(args.prompts, args.batch, args.seed)
+    else:
+        out = generation(args.tokens, args.seed)
     print(json.dumps(out))
 
 

@@ -22,3 +22,11 @@ def test_dataset_sweep_small():
         assert out[key]["tokens_per_s"] > 0.0
     # with a lognormal length mix, padding to the batch maximum in arrival order wastes the most
     assert out["speedup_vs_arrival_order"] > 1.0
+
+
+def test_generation_sweep_small():
+    from paper_2404_09529_b200 import sweep
+    out = sweep.generation(n_tokens=3, seed=1)
+    toy = out["toy_9x1_1x1000"]
+    assert toy["cached_tokens"] == 1009 and toy["padded_cached_tokens"] == 10000
+    assert toy["ms_per_token"] > 0.0 and toy["ms_per_token_padded"] > 0.0
