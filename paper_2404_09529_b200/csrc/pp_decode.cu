@@ -75,23 +75,25 @@ decode_append_kernel(const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat1
   }
 }
 
-// partial results: [chunk][query head][D + 2] floats = (m, l, o[D]), m in scaled log2 units
-template <int D>
+// partial results: [chunk][query head][D + 2] floats = (m, l, o[D]), m in scaled log2 units.
+// G: compile-time bound on the query heads per KV head (1, 2, 4 or 8), so that a small group does
+// not pay registers for a large one.
+template <int D, int G>
 __global__ void __launch_bounds__(kDecodeThreads)
 decode_partial_kernel(const __nv_bfloat16* __restrict__ q_rot, const __nv_bfloat16* __restrict__ k_cache,
                       const __nv_bfloat16* __restrict__ v_cache, float* __restrict__ partial,
                       const int32_t* __restrict__ table, DecodeTable T, int32_t n_q_heads, int32_t n_kv_heads,
                       int32_t group, float scale_log2) {
   constexpr int E = D / 32;                       // elements of a row per lane
-  __shared__ float s_m[4][kMaxGroup], s_l[4][kMaxGroup], s_o[4][kMaxGroup][D];
+  __shared__ float s_m[4][G], s_l[4][G], s_o[4][G][D];
   const int chunk = blockIdx.x, kvh = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int i = table[T.chunks + 3 * chunk], key0 = table[T.chunks + 3 * chunk + 1], n_keys = table[T.chunks + 3 * chunk + 2];
   const int64_t cap = table[T.cache_cap + i];
   const int64_t base = reinterpret_cast<const int64_t*>(table + T.cache_off)[i] + (int64_t)kvh * cap * D;
-  float q[kMaxGroup][E], acc[kMaxGroup][E], m[kMaxGroup], l[kMaxGroup];
+  float q[G][E], acc[G][E], m[G], l[G];
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) {
+  for (int h = 0; h < G; ++h) {
     m[h] = -INFINITY;
     l[h] = 0.f;
 #pragma unroll
@@ -100,7 +102,7 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q_rot, const __nv_bfloat
       q[h][e] = (h < group) ? __bfloat162float(q_rot[((int64_t)i * n_q_heads + kvh * group + h) * D + lane * E + e]) : 0.f;
     }
   }
-  // one 4- or 8-byte load per lane and row; two keys per iteration keep four loads in flight
+  // one 4- or 8-byte load per lane and row; four keys per iteration keep eight loads in flight
   auto load_row = [&](const __nv_bfloat16* p, float (&out)[E]) {
     if constexpr (E == 4) {
       const uint2 u = __ldg(reinterpret_cast<const uint2*>(p));
@@ -115,7 +117,7 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q_rot, const __nv_bfloat
   };
   auto one_key = [&](const float (&kk)[E], const float (&vv)[E]) {
 #pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h) {
+    for (int h = 0; h < G; ++h) {
       if (h >= group) break;
       float s = 0.f;
 #pragma unroll
@@ -134,14 +136,15 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q_rot, const __nv_bfloat
   const __nv_bfloat16* kbase = k_cache + base + (int64_t)key0 * D + lane * E;
   const __nv_bfloat16* vbase = v_cache + base + (int64_t)key0 * D + lane * E;
   int t = warp;
-  for (; t + 4 < n_keys; t += 8) {
-    float k0[E], v0[E], k1[E], v1[E];
-    load_row(kbase + (int64_t)t * D, k0);
-    load_row(vbase + (int64_t)t * D, v0);
-    load_row(kbase + (int64_t)(t + 4) * D, k1);
-    load_row(vbase + (int64_t)(t + 4) * D, v1);
-    one_key(k0, v0);
-    one_key(k1, v1);
+  for (; t + 12 < n_keys; t += 16) {
+    float kx[4][E], vx[4][E];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      load_row(kbase + (int64_t)(t + 4 * u) * D, kx[u]);
+      load_row(vbase + (int64_t)(t + 4 * u) * D, vx[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) one_key(kx[u], vx[u]);
   }
   for (; t < n_keys; t += 4) {
     float k0[E], v0[E];
@@ -151,7 +154,7 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q_rot, const __nv_bfloat
   }
   // merge the four warps
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) {
+  for (int h = 0; h < G; ++h) {
     if (h >= group) break;
     if (lane == 0) { s_m[warp][h] = m[h]; s_l[warp][h] = l[h]; }
 #pragma unroll
@@ -293,16 +296,20 @@ extern "C" int pp_decode_step(const pp_attn_params* params, const int32_t* lengt
   const float scale_log2 = scale * 1.4426950408889634f;
   const int group = params->n_q_heads / params->n_kv_heads;
   const dim3 grid_p((unsigned)L.n_chunks, (unsigned)params->n_kv_heads), grid_c((unsigned)k, (unsigned)params->n_q_heads);
+#define PP_DECODE_PARTIAL(DD, GG)                                                                                \
+  pp::decode_partial_kernel<DD, GG><<<grid_p, pp::kDecodeThreads, 0, s>>>(                                       \
+      q_rot, (const __nv_bfloat16*)k_cache, (const __nv_bfloat16*)v_cache, partial, d_table, L.T,                \
+      params->n_q_heads, params->n_kv_heads, group, scale_log2)
 #define PP_DECODE_LAUNCH(DD)                                                                                     \
   pp::decode_append_kernel<DD><<<k, pp::kDecodeThreads, 0, s>>>(                                                 \
       (const __nv_bfloat16*)q_new, (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, q_rot,              \
       (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table, L.T, params->n_q_heads, params->n_kv_heads, freq); \
-  pp::decode_partial_kernel<DD><<<grid_p, pp::kDecodeThreads, 0, s>>>(                                           \
-      q_rot, (const __nv_bfloat16*)k_cache, (const __nv_bfloat16*)v_cache, partial, d_table, L.T,                \
-      params->n_q_heads, params->n_kv_heads, group, scale_log2);                                                 \
+  if (group == 1) PP_DECODE_PARTIAL(DD, 1); else if (group == 2) PP_DECODE_PARTIAL(DD, 2);                       \
+  else if (group <= 4) PP_DECODE_PARTIAL(DD, 4); else PP_DECODE_PARTIAL(DD, 8);                                  \
   pp::decode_combine_kernel<DD><<<grid_c, DD, 0, s>>>(partial, (__nv_bfloat16*)o, d_table, L.T, params->n_q_heads)
   if (params->head_dim == 128) { PP_DECODE_LAUNCH(128); } else { PP_DECODE_LAUNCH(64); }
 #undef PP_DECODE_LAUNCH
+#undef PP_DECODE_PARTIAL
   e = cudaGetLastError();
   return e == cudaSuccess ? PP_OK : pp::note_cuda_error((int)e, "decode kernel launch");
 }
