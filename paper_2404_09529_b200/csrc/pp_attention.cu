@@ -344,6 +344,24 @@ __device__ __forceinline__ void ring_write(volatile int* e, int w, const Work& w
 enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWaitKFull, kWaitKEmpty,
                 kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty, kWaitPair, kWaitEpilogue, kWaitRowSum };
 
+// Start row of the prompt that holds bin-local row `i_row`, among the prompts seg_begin .. seg_end-1
+// of a bin whose start rows (ascending) are in `starts`; `lo` if none of them starts at or before the
+// row. All 32 lanes call it with the same range: the starts are loaded 32 at a time, one per lane,
+// and handed round with shuffles, so the walk costs one memory round trip per 32 prompts.
+__device__ __forceinline__ int seg_start_at(const int32_t* starts, int seg_begin, int seg_end, int i_row, int lo, int lane) {
+  const int row_max = i_row - lane + 31;               // the warp's rows are consecutive
+  for (int base = seg_begin; base < seg_end; base += 32) {
+    const int cnt = min(32, seg_end - base);
+    const int mine = (lane < cnt) ? __ldg(starts + base + lane) : 0x7fffffff;
+    for (int sg = 0; sg < cnt; ++sg) {
+      const int st = __shfl_sync(0xffffffffu, mine, sg);
+      if (st > row_max) return lo;                     // warp-uniform: no later prompt starts in these rows
+      if (st <= i_row) lo = st;
+    }
+  }
+  return lo;
+}
+
 // kIndep = false: the two slots of a CTA work on one item and share its K/V stream (long
 //   sequences, GQA head pairs). kIndep = true: every slot draws its own single-tile items and loads
 //   its own K/V tiles (64 rows each), so neither slot ever waits for the other (short prompts, where
@@ -388,7 +406,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const uint32_t bar_q_rot = s_misc + 384;       // [2] Q_t has been rotated in place (fused path)
   const uint32_t bar_pair0 = s_misc + 896;       // [2 slots][4 quadrants] rendezvous of the two warps that share rows
   const uint32_t bar_epi0 = s_misc + 960;        // [2] rendezvous of a slot's 128 epilogue threads
-  const uint32_t bar_l_ready = s_misc + 976;     // [2] independent mode: the slot's row sums are in shared memory
+  const uint32_t bar_l_ready = s_misc + 976;     // [2][2] independent mode: the slot's row sums of item i are in shared memory ([slot][i & 1])
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 400);
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 404);
   volatile int* s_ring = reinterpret_cast<volatile int*>(misc + 416);   // [2 rings][kRing][kRingInts]
@@ -418,7 +436,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_init(bar_o_full + 8 * i, 1);
       mbar_init(bar_o_empty + 8 * i, kIndep ? kSoftmaxThreads / 2 : kSoftmaxThreads);
       mbar_init(bar_epi0 + 8 * i, kSoftmaxThreads / 2);
-      mbar_init(bar_l_ready + 8 * i, kSoftmaxThreads / 2);
+      mbar_init(bar_l_ready + 16 * i, kSoftmaxThreads / 2);
+      mbar_init(bar_l_ready + 16 * i + 8, kSoftmaxThreads / 2);
       for (int qd = 0; qd < 4; ++qd) mbar_init(bar_pair0 + 8 * (4 * i + qd), 64);
     }
     for (int s = 0; s < NK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
@@ -764,20 +783,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       volatile float* x_l = s_xchg + t * 128 + row;            // + 256 * (item & 1)
       bool ok = true;
       // key range [key_lo, key_hi] of this thread's row from a ring entry (empty for padding rows)
+      // (all lanes of the warp call it together: the prompts' start rows are loaded once per warp)
       auto row_range = [&](const volatile int* e, int& key_lo, int& key_hi) {
         const int i_row = e[4] + row;
-        key_lo = 1; key_hi = 0;
-        if (i_row < e[12]) {
-          key_lo = e[14];
-          if (!(e[18] & 1)) {                          // several prompts in this tile: walk their starts
-            for (int sg = e[16] + 1; sg < e[13]; ++sg) {
-              const int st = __ldg(tb + args.off_seg_start + sg);
-              if (st > i_row) break;
-              key_lo = st;
-            }
-          }
-          key_hi = i_row;
-        }
+        int lo = e[14];
+        if (!(e[18] & 1)) lo = seg_start_at(tb + args.off_seg_start, e[16] + 1, e[13], i_row, lo, lane);
+        const bool real = i_row < e[12];
+        key_lo = real ? lo : 1;
+        key_hi = real ? i_row : 0;
       };
       if (h == 0) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxIndep));
@@ -921,9 +934,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ++tcount;
           }
           if (!ok) break;
-          // hand the row sum to the helper thread of this row (arrive has release semantics)
+          // The row sum goes to the helper thread of this row (arrive has release semantics). The
+          // softmax threads can finish item i+1 before the helpers have picked up item i, but not
+          // item i+2 (its scores are issued after the epilogue of item i has read O_t), so the
+          // hand-over is double-buffered by item parity, barrier included.
           x_l[256 * (it_n & 1u)] = l_run;
-          mbar_arrive(bar_l_ready + 8 * t);
+          mbar_arrive(bar_l_ready + 16 * t + 8 * (it_n & 1u));
           PROF_LAP(7);
           ++it_n;
         }
@@ -1003,7 +1019,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const uint32_t pi = it_n - 1u;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full + 8 * t, pi & 1u, wctx, kWaitOFull));
             if (!ok) break;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_l_ready + 8 * t, pi & 1u, wctx, kWaitRowSum));
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_l_ready + 16 * t + 8 * (pi & 1u), (pi >> 1) & 1u, wctx, kWaitRowSum));
             if (!ok) break;
             tc_fence_after();
             const float l_row = x_l[256 * (pi & 1u)];
@@ -1134,22 +1150,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const bool used = jb_t < je_t;
       const int i_row = q_row0_t + row;                // bin-local query row
       int key_lo = 1, key_hi = 0;                      // visible keys [key_lo, key_hi]; empty for padding
-      if (used && i_row < bin_used) {
-        key_lo = key_lo_t;
-        if (!(single_seg & 1)) {                       // several prompts in this tile: walk their starts
-          for (int sg = seg_first_t + 1; sg < seg_end; ++sg) {
-            const int st = __ldg(tb + args.off_seg_start + sg);
-            if (st > i_row) break;
-            key_lo = st;
-          }
-        }
-        key_hi = i_row;
+      if (used) {                                      // warp-uniform
+        int lo = key_lo_t;
+        if (!(single_seg & 1))                         // several prompts in this tile: find this row's
+          lo = seg_start_at(tb + args.off_seg_start, seg_first_t + 1, seg_end, i_row, lo, lane);
+        if (i_row < bin_used) { key_lo = lo; key_hi = i_row; }
       }
       PROF_LAP(8);
-      // Fused path: Q arrives raw and is rotated in shared memory. In independent mode the rotation
-      // of item i+1 was already done before the epilogue of item i (see below), except for the
-      // first item.
-      if (args.rope_table && (!kIndep || it_n == 0)) {
+      // Fused path: Q arrives raw and is rotated in shared memory.
+      if (args.rope_table) {
         ok = rotate_q(used ? key_hi - key_lo : -1, it_n & 1u);
         if (!ok) break;
         PROF_LAP(11);
@@ -1297,33 +1306,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       if (!ok) break;
 
-      if (kIndep && args.rope_table) {
-        PROF_LAP(5);
-        // Independent mode, fused path: while this item's last P V product is still running, get the
-        // next item's Q ready, so that its first S tile is computed under this item's epilogue.
-        const uint32_t nring = (uint32_t)t * kRing + (it_n + 1) % kRing;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * nring, ((it_n + 1) / kRing) & 1u, wctx, kWaitItemFull));
-        if (!ok) break;
-        const volatile int* ne = s_ring + nring * kRingInts;   // peeked, not consumed here
-        if (ne[0] >= 0) {
-          const int n_row = ne[4] + row;
-          int n_pos = -1;
-          if (n_row < ne[12]) {
-            int n_lo = ne[14];
-            if (!(ne[18] & 1)) {
-              for (int sg = ne[16] + 1; sg < ne[13]; ++sg) {
-                const int st = __ldg(tb + args.off_seg_start + sg);
-                if (st > n_row) break;
-                n_lo = st;
-              }
-            }
-            n_pos = n_row - n_lo;
-          }
-          ok = rotate_q(n_pos, (it_n + 1) & 1u);
-          if (!ok) break;
-          PROF_LAP(11);
-        }
-      }
       // epilogue: O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store
       PROF_LAP(5);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full + 8 * t, it_n & 1u, wctx, kWaitOFull));
