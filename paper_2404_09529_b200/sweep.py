@@ -1,4 +1,4 @@
-"""Two measurement sweeps over the prefill path, on synthetic batches (Sections 5.2 and 6 of the paper).
+"""Measurement sweeps over the prefill and decode paths, on synthetic batches (Sections 5.2, 6 and 7 of the paper).
 
 ``predictor``: batches of k prompts with lengths uniform in [1, 512]; for every batch the packed
 and the padded (full-batching) path are timed and the speedup is regressed on the two batch
@@ -14,11 +14,17 @@ tokens per second of each schedule.
 token and one of 1000 tokens, 20 generated tokens), against the same steps with every prompt
 declared as long as the longest (what padded caches cost).
 
+``shapes``: batches of 16 prompts whose lengths follow lognormal distributions fitted to the
+minimum / mean / maximum prompt length the paper reports for each of its six evaluation sets
+(appendix table of dataset length statistics; lengths only, no text), on the attention-layer shapes
+of the 1.3 B and 7 B models of its model table: packed against padded path, per length profile.
+
 Each prints one JSON object. They only marshal arguments: all arithmetic runs in the library.
 
     python -m paper_2404_09529_b200.sweep predictor [--batches 40] [--k 16]
     python -m paper_2404_09529_b200.sweep dataset [--prompts 4096] [--batch 16]
     python -m paper_2404_09529_b200.sweep generation [--tokens 20]
+    python -m paper_2404_09529_b200.sweep shapes [--batches 8] [--k 16]
 """
 from __future__ import annotations
 
@@ -154,6 +160,56 @@ def generation(n_tokens: int, seed: int) -> dict:
     return out
 
 
+# Length profiles: (mu, sigma) of ln(length) fitted to the reported mean, clipped to the reported
+# [min, max] of each evaluation set.
+LENGTH_PROFILES = {
+    "wiki256": (4.195, 0.437, 1, 256),
+    "wiki512": (4.656, 0.512, 6, 512),
+    "mmlu": (3.525, 1.126, 4, 1102),
+    "hh_rlhf": (5.275, 0.684, 22, 1620),
+    "alpaca": (4.709, 0.504, 43, 527),
+    "samsum": (4.939, 0.618, 21, 942),
+}
+# attention-layer shapes (query heads, KV heads, head_dim): hidden 2048 / 16 heads and 4096 / 32 heads
+LAYER_SHAPES = {"1.3b": (16, 16, 128), "7b": (32, 32, 128)}
+
+
+def shapes(n_batches: int, k: int, seed: int) -> dict:
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    out = {"sweep": "shapes", "k": k, "batches": n_batches,
+           "lengths": "lognormal fitted to each evaluation set's reported min / mean / max", "profiles": {}}
+    for pname, (mu, sigma, lo, hi) in LENGTH_PROFILES.items():
+        rng = np.random.default_rng(seed)
+        batches = [np.clip(np.rint(np.exp(mu + sigma * rng.standard_normal(k))), lo, hi).astype(np.int32)
+                   for _ in range(n_batches)]
+        row = {"mean_length": float(np.mean([b.mean() for b in batches])),
+               "mean_bins": None, "models": {}}
+        for mname, (hq, hkv, d) in LAYER_SHAPES.items():
+            ms_packed = ms_padded = 0.0
+            bins = 0
+            for lengths in batches:
+                t = int(lengths.sum())
+                q = torch.randn(t, hq, d, generator=gen, device="cuda").to(torch.bfloat16)
+                kk = torch.randn(t, hkv, d, generator=gen, device="cuda").to(torch.bfloat16)
+                v = torch.randn(t, hkv, d, generator=gen, device="cuda").to(torch.bfloat16)
+                for mode in ("packed", "padded"):
+                    b = PrefillBatch(lengths, hq, hkv, d, BASE, mode=mode)
+                    b.load(q, kk, v)
+                    ms = _time_ms(lambda: b.run_fused(repack=True))
+                    assert b.device_status() == 0
+                    if mode == "packed":
+                        ms_packed += ms
+                        bins += int(b.pack.n_bins)
+                    else:
+                        ms_padded += ms
+                    del b
+            row["mean_bins"] = bins / n_batches
+            row["models"][mname] = {"ms_packed": ms_packed / n_batches, "ms_padded": ms_padded / n_batches,
+                                    "speedup": ms_padded / ms_packed}
+        out["profiles"][pname] = row
+    return out
+
+
 def main() -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -168,6 +224,10 @@ def main() -> None:
     gsub = sub.add_parser("generation")
     gsub.add_argument("--tokens", type=int, default=20)
     gsub.add_argument("--seed", type=int, default=0)
+    ssub = sub.add_parser("shapes")
+    ssub.add_argument("--batches", type=int, default=8)
+    ssub.add_argument("--k", type=int, default=16)
+    ssub.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("the sweeps need a GPU: the library has no CPU path")
@@ -175,8 +235,10 @@ def main() -> None:
         out = predictor(args.batches, args.k, args.seed)
     elif args.cmd == "dataset":
         out = dataset(args.prompts, args.batch, args.seed)
-    else:
+    elif args.cmd == "generation":
         out = generation(args.tokens, args.seed)
+    else:
+        out = shapes(args.batches, args.k, args.seed)
     print(json.dumps(out))
 
 

@@ -1,4 +1,4 @@
-"""The two measurement sweeps run end to end on small inputs (GPU only: the library has no CPU path)."""
+"""The measurement sweeps run end to end on small inputs (GPU only: the library has no CPU path)."""
 import pytest
 
 pytestmark = pytest.mark.gpu
@@ -30,3 +30,14 @@ def test_generation_sweep_small():
     toy = out["toy_9x1_1x1000"]
     assert toy["cached_tokens"] == 1009 and toy["padded_cached_tokens"] == 10000
     assert toy["ms_per_token"] > 0.0 and toy["ms_per_token_padded"] > 0.0
+
+
+def test_shapes_sweep_small():
+    from paper_2404_09529_b200 import sweep
+    out = sweep.shapes(n_batches=1, k=8, seed=1)
+    assert set(out["profiles"]) == set(sweep.LENGTH_PROFILES)
+    for name, row in out["profiles"].items():
+        lo, hi = sweep.LENGTH_PROFILES[name][2:]
+        assert lo <= row["mean_length"] <= hi and 1 <= row["mean_bins"] <= 8
+        for model in sweep.LAYER_SHAPES:
+            assert row["models"][model]["ms_packed"] > 0.0 and row["models"][model]["ms_padded"] > 0.0
