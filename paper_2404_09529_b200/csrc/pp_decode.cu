@@ -56,22 +56,56 @@ decode_append_kernel(const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat1
     s_sin[threadIdx.x] = sn;
   }
   __syncthreads();
-  // (head, j) pairs of q, then of k; v is copied as it is
-  for (int u = threadIdx.x; u < (n_q_heads + n_kv_heads) * kHalf; u += kDecodeThreads) {
-    const int head = u / kHalf, j = u - head * kHalf;
-    const bool is_k = head >= n_q_heads;
-    const __nv_bfloat16* src = is_k ? k_new + ((int64_t)i * n_kv_heads + (head - n_q_heads)) * D
-                                    : q_new + ((int64_t)i * n_q_heads + head) * D;
-    __nv_bfloat16* dst = is_k ? k_cache + base + ((int64_t)(head - n_q_heads) * cap + pos) * D
-                              : q_rot + ((int64_t)i * n_q_heads + head) * D;
-    const float a = __bfloat162float(src[j]), b = __bfloat162float(src[j + kHalf]);
-    const float c = s_cos[j], s = s_sin[j];
-    dst[j] = __float2bfloat16_rn(__fmaf_rn(a, c, -__fmul_rn(b, s)));
-    dst[j + kHalf] = __float2bfloat16_rn(__fmaf_rn(b, c, __fmul_rn(a, s)));
+  // Units of eight (j, j + D/2) pairs: (head, group of eight j) of q, then of k. 16-byte accesses, and
+  // the loads of up to four units are issued before the first store (the compiler cannot prove
+  // that the destinations do not alias the sources, so it would serialise them otherwise).
+  constexpr int kGroups = kHalf / 8;
+  const int n_units = (n_q_heads + n_kv_heads) * kGroups;
+  for (int u0 = threadIdx.x; u0 < n_units; u0 += 4 * kDecodeThreads) {
+    uint4 lo[4], hi[4];
+    __nv_bfloat16* dst[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const int u = u0 + x * kDecodeThreads;
+      dst[x] = nullptr;
+      if (u < n_units) {
+        const int head = u / kGroups, g = u - head * kGroups;
+        const bool is_k = head >= n_q_heads;
+        const __nv_bfloat16* src = is_k ? k_new + ((int64_t)i * n_kv_heads + (head - n_q_heads)) * D
+                                        : q_new + ((int64_t)i * n_q_heads + head) * D;
+        dst[x] = (is_k ? k_cache + base + ((int64_t)(head - n_q_heads) * cap + pos) * D
+                       : q_rot + ((int64_t)i * n_q_heads + head) * D) + 8 * g;
+        lo[x] = __ldg(reinterpret_cast<const uint4*>(src + 8 * g));
+        hi[x] = __ldg(reinterpret_cast<const uint4*>(src + 8 * g + kHalf));
+      }
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      if (!dst[x]) continue;
+      const int j0 = (int)((u0 + x * kDecodeThreads) % kGroups) * 8;
+      uint32_t* l32 = reinterpret_cast<uint32_t*>(&lo[x]);
+      uint32_t* h32 = reinterpret_cast<uint32_t*>(&hi[x]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&l32[e]));
+        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&h32[e]));
+        const float c0 = s_cos[j0 + 2 * e], s0 = s_sin[j0 + 2 * e], c1 = s_cos[j0 + 2 * e + 1], s1 = s_sin[j0 + 2 * e + 1];
+        const __nv_bfloat162 lo2 = __floats2bfloat162_rn(__fmaf_rn(a.x, c0, -__fmul_rn(b.x, s0)),
+                                                         __fmaf_rn(a.y, c1, -__fmul_rn(b.y, s1)));
+        const __nv_bfloat162 hi2 = __floats2bfloat162_rn(__fmaf_rn(b.x, c0, __fmul_rn(a.x, s0)),
+                                                         __fmaf_rn(b.y, c1, __fmul_rn(a.y, s1)));
+        l32[e] = *reinterpret_cast<const uint32_t*>(&lo2);
+        h32[e] = *reinterpret_cast<const uint32_t*>(&hi2);
+      }
+      *reinterpret_cast<uint4*>(dst[x]) = lo[x];
+      *reinterpret_cast<uint4*>(dst[x] + kHalf) = hi[x];
+    }
   }
-  for (int u = threadIdx.x; u < n_kv_heads * D; u += kDecodeThreads) {
-    const int head = u / D, e = u - head * D;
-    v_cache[base + ((int64_t)head * cap + pos) * D + e] = v_new[((int64_t)i * n_kv_heads + head) * D + e];
+  // v is copied as it is
+  for (int u = threadIdx.x; u < n_kv_heads * (D / 8); u += kDecodeThreads) {
+    const int head = u / (D / 8), g = u - head * (D / 8);
+    *reinterpret_cast<uint4*>(v_cache + base + ((int64_t)head * cap + pos) * D + 8 * g) =
+        __ldg(reinterpret_cast<const uint4*>(v_new + ((int64_t)i * n_kv_heads + head) * D + 8 * g));
   }
 }
 
