@@ -3,7 +3,7 @@
 // keys and values every prompt has. Three kernels:
 //   decode_append_kernel     rotates the new token's q and k by its position (= tokens cached so far),
 //                            appends k' and v to the prompt's caches, leaves q' in the workspace
-//   decode_partial_kernel    one CTA per (chunk of 256 cached keys, KV head): scores, online softmax
+//   decode_partial_kernel    one CTA per (chunk of 256 or 64 cached keys, KV head): scores, online softmax
 //                            and P V for the query heads of that KV head, partial (m, l, o) out
 //   decode_combine_kernel    merges a prompt's chunks into o
 // HBM-bound: K and V of every cached token are read once.
@@ -229,11 +229,15 @@ decode_combine_kernel(const float* __restrict__ partial, __nv_bfloat16* __restri
   o[((int64_t)i * n_q_heads + head) * D + d] = __float2bfloat16_rn(oo / ll);
 }
 
-constexpr int kChunkKeys = 256;
+// Keys per chunk: 256 when that already gives every SM several CTAs, else 64, so that a small batch
+// (a few prompts, one of them long) is spread over more CTAs and each warp's chain of dependent row
+// loads is a quarter as long.
+constexpr int kChunkKeysLarge = 256, kChunkKeysSmall = 64;
+constexpr int64_t kChunkCtasWanted = 148 * 8;
 
-int64_t count_chunks(const int32_t* lengths, int32_t k) {
+int64_t count_chunks(const int32_t* lengths, int32_t k, int chunk_keys) {
   int64_t n = 0;
-  for (int32_t i = 0; i < k; ++i) n += ((int64_t)lengths[i] + 1 + kChunkKeys - 1) / kChunkKeys;
+  for (int32_t i = 0; i < k; ++i) n += ((int64_t)lengths[i] + 1 + chunk_keys - 1) / chunk_keys;
   return n;
 }
 size_t up4(size_t x) { return (x + 3) & ~size_t(3); }
@@ -242,10 +246,16 @@ struct DecodeLayout {
   DecodeTable T;
   size_t table_ints, q_rot_bytes_off, partial_bytes_off, total_bytes;
   int64_t n_chunks;
+  int chunk_keys;
 };
 DecodeLayout decode_layout(const pp_attn_params& p, const int32_t* lengths, int32_t k) {
   DecodeLayout L;
-  L.n_chunks = count_chunks(lengths, k);
+  L.chunk_keys = kChunkKeysLarge;
+  L.n_chunks = count_chunks(lengths, k, L.chunk_keys);
+  if (L.n_chunks * p.n_kv_heads < kChunkCtasWanted) {
+    L.chunk_keys = kChunkKeysSmall;
+    L.n_chunks = count_chunks(lengths, k, L.chunk_keys);
+  }
   size_t off = 0;
   L.T.chunks = (int32_t)off; off += up4(3 * (size_t)L.n_chunks);
   L.T.chunk_ptr = (int32_t)off; off += up4((size_t)k + 1);
@@ -306,10 +316,10 @@ extern "C" int pp_decode_step(const pp_attn_params* params, const int32_t* lengt
   for (int32_t i = 0; i < k; ++i) {
     h[L.T.chunk_ptr + i] = c;
     const int32_t n = lengths[i] + 1;                     // the new token is attended too
-    for (int32_t key0 = 0; key0 < n; key0 += pp::kChunkKeys, ++c) {
+    for (int32_t key0 = 0; key0 < n; key0 += L.chunk_keys, ++c) {
       h[L.T.chunks + 3 * c] = i;
       h[L.T.chunks + 3 * c + 1] = key0;
-      h[L.T.chunks + 3 * c + 2] = n - key0 < pp::kChunkKeys ? n - key0 : pp::kChunkKeys;
+      h[L.T.chunks + 3 * c + 2] = n - key0 < L.chunk_keys ? n - key0 : L.chunk_keys;
     }
     h[L.T.lengths + i] = lengths[i];
     h[L.T.cache_cap + i] = cache_cap[i];

@@ -21,6 +21,8 @@ def _case(lengths, hq, hkv, d, seed):
     (np.array([1, 1, 1, 1000, 1, 1, 1, 1, 1, 1], np.int32), 8, 8, 128, 10000.0),   # the paper's toy mix
     (np.array([300, 17, 255, 256, 257, 64], np.int32), 8, 2, 128, 500000.0),
     (np.array([40, 9, 513], np.int32), 4, 4, 64, 10000.0),
+    # enough (chunk, KV head) pairs for the 256-key chunks (smaller batches run 64-key chunks)
+    (np.array([255, 256, 257, 511, 512, 513, 767, 768, 300, 64, 1000, 129] * 4, np.int32), 16, 16, 64, 10000.0),
 ])
 def test_decode_steps_match_oracle(lengths, hq, hkv, d, base):
     from paper_2404_09529_b200.runner import DecodeBatch, PrefillBatch
