@@ -342,7 +342,7 @@ __device__ __forceinline__ void ring_write(volatile int* e, int w, const Work& w
 }
 
 enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWaitKFull, kWaitKEmpty,
-                kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty, kWaitPair, kWaitEpilogue, kWaitRowSum };
+                kWaitVFull, kWaitVEmpty, kWaitS, kWaitP, kWaitOFull, kWaitOEmpty, kWaitPair, kWaitRowSum };
 
 // Start row of the prompt that holds bin-local row `i_row`, among the prompts seg_begin .. seg_end-1
 // of a bin whose start rows (ascending) are in `starts`; `lo` if none of them starts at or before the
@@ -405,7 +405,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   const uint32_t bar_v_empty = s_misc + 352;     // [4]
   const uint32_t bar_q_rot = s_misc + 384;       // [2] Q_t has been rotated in place (fused path)
   const uint32_t bar_pair0 = s_misc + 896;       // [2 slots][4 quadrants] rendezvous of the two warps that share rows
-  const uint32_t bar_epi0 = s_misc + 960;        // [2] rendezvous of a slot's 128 epilogue threads
   const uint32_t bar_l_ready = s_misc + 976;     // [2][2] independent mode: the slot's row sums of item i are in shared memory ([slot][i & 1])
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(misc + 400);
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 404);
@@ -435,7 +434,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       mbar_init(bar_o_full + 8 * i, 1);
       mbar_init(bar_o_empty + 8 * i, kIndep ? kSoftmaxThreads / 2 : kSoftmaxThreads);
-      mbar_init(bar_epi0 + 8 * i, kSoftmaxThreads / 2);
       mbar_init(bar_l_ready + 16 * i, kSoftmaxThreads / 2);
       mbar_init(bar_l_ready + 16 * i + 8, kSoftmaxThreads / 2);
       for (int qd = 0; qd < 4; ++qd) mbar_init(bar_pair0 + 8 * (4 * i + qd), 64);
@@ -949,14 +947,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #endif
       } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsHelper));
-        const uint32_t bar_epi = bar_epi0 + 8 * (uint32_t)t;
-        uint32_t epi_ph = 0;
-        auto rendezvous = [&](const uint32_t bar, uint32_t& ph, const int code) -> bool {
-          mbar_arrive(bar);
-          const bool r = __all_sync(0xffffffffu, mbar_wait(bar, ph, wctx, code));
-          ph ^= 1u;
-          return r;
-        };
         uint32_t it_n = 0;
         int p_q_row0 = 0, p_head = 0, p_bin = 0;         // coordinates of the previous item (its epilogue is due)
         while (true) {
@@ -1024,13 +1014,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tc_fence_after();
             const float l_row = x_l[256 * (pi & 1u)];
             const float inv_l = l_row > 0.f ? 1.f / l_row : 0.f;
-            const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes;
-            const uint32_t stage_row = stage + (uint32_t)row * 128;
+            // Each warp stages and stores its own 32 rows (a 32-row TMA box), so the epilogue needs
+            // no rendezvous between warps: lane 0 issues the warp's stores and is the one to wait
+            // until the previous store has read the staging rows.
+            const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes + (uint32_t)quad * (32 * 128);
+            const uint32_t stage_row = stage + (uint32_t)lane * 128;
+            const int p_row0 = p_q_row0 + 32 * quad;
 #pragma unroll 1
             for (int hh = 0; hh < D / 64; ++hh) {          // 64 columns (one TMA box) at a time
-              // the staging buffer is free once the previous store has read it
-              if (row == 0) tma_store_wait_read();
-              if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
+              if (lane == 0) tma_store_wait_read();
+              __syncwarp();
               uint32_t ov[64];
               tmem_ld32(tmem_o + hh * 64, *reinterpret_cast<uint32_t(*)[32]>(&ov[0]));
               tmem_ld32(tmem_o + hh * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[32]));
@@ -1041,7 +1034,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               }
 #pragma unroll
               for (int c16 = 0; c16 < 8; ++c16) {
-                const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)row & 7u)) << 4);
+                const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)lane & 7u)) << 4);
                 const uint32_t w0 = pack_bf16(__uint_as_float(ov[c16 * 8 + 0]) * inv_l, __uint_as_float(ov[c16 * 8 + 1]) * inv_l);
                 const uint32_t w1 = pack_bf16(__uint_as_float(ov[c16 * 8 + 2]) * inv_l, __uint_as_float(ov[c16 * 8 + 3]) * inv_l);
                 const uint32_t w2 = pack_bf16(__uint_as_float(ov[c16 * 8 + 4]) * inv_l, __uint_as_float(ov[c16 * 8 + 5]) * inv_l);
@@ -1049,9 +1042,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
               }
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-              if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
-              if (row == 0) {
-                tma_store_4d(&map_o, stage, hh * 64, p_head, p_q_row0, p_bin);
+              __syncwarp();
+              if (lane == 0 && p_row0 < args.capacity) {
+                tma_store_4d(&map_o, stage, hh * 64, p_head, p_row0, p_bin);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
               }
             }
@@ -1061,7 +1054,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           p_q_row0 = c_q_row0; p_head = c_head; p_bin = c_bin;
           ++it_n;
         }
-        if (row == 0) tma_store_wait_read();     // staging must outlive the last store's read
+        if (lane == 0) tma_store_wait_read();    // staging must outlive the last store's read
       }
     } else {
     // ---------------------------------------------------------------- shared-stream mode
@@ -1073,8 +1066,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // Rendezvous points are mbarriers (arrive, then a bounded wait) rather than named barriers, so
     // that a warp whose partner gave up on a wait cannot be left waiting for it.
     const uint32_t bar_pair = bar_pair0 + 8 * (uint32_t)(t * 4 + quad);
-    const uint32_t bar_epi = bar_epi0 + 8 * (uint32_t)t;
-    uint32_t pair_ph = 0, epi_ph = 0;
+    uint32_t pair_ph = 0;
     auto rendezvous = [&](const uint32_t bar, uint32_t& ph, const int code) -> bool {
       mbar_arrive(bar);
       const bool r = __all_sync(0xffffffffu, mbar_wait(bar, ph, wctx, code));
@@ -1322,13 +1314,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (h == 0) {
           tc_fence_after();
           const float inv_l = l_row > 0.f ? 1.f / l_row : 0.f;
-          const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes;
-          const uint32_t stage_row = stage + (uint32_t)row * 128;
+          // each warp stages and stores its own 32 rows (a 32-row TMA box): no rendezvous between
+          // warps; lane 0 issues the warp's stores and waits for the previous one to have read the rows
+          const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes + (uint32_t)quad * (32 * 128);
+          const uint32_t stage_row = stage + (uint32_t)lane * 128;
+          const int row0_w = q_row0_t + 32 * quad;
 #pragma unroll 1
           for (int hh = 0; hh < D / 64; ++hh) {          // 64 columns (one TMA box) at a time
-            // the staging buffer is free once the previous store has read it
-            if (row == 0) tma_store_wait_read();
-            if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
+            if (lane == 0) tma_store_wait_read();
+            __syncwarp();
             uint32_t ov[64];
             tmem_ld32(tmem_o + hh * 64, *reinterpret_cast<uint32_t(*)[32]>(&ov[0]));
             tmem_ld32(tmem_o + hh * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[32]));
@@ -1339,7 +1333,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
 #pragma unroll
             for (int c16 = 0; c16 < 8; ++c16) {
-              const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)row & 7u)) << 4);
+              const uint32_t addr = stage_row + (((uint32_t)c16 ^ ((uint32_t)lane & 7u)) << 4);
               const uint32_t w0 = pack_bf16(__uint_as_float(ov[c16 * 8 + 0]) * inv_l, __uint_as_float(ov[c16 * 8 + 1]) * inv_l);
               const uint32_t w1 = pack_bf16(__uint_as_float(ov[c16 * 8 + 2]) * inv_l, __uint_as_float(ov[c16 * 8 + 3]) * inv_l);
               const uint32_t w2 = pack_bf16(__uint_as_float(ov[c16 * 8 + 4]) * inv_l, __uint_as_float(ov[c16 * 8 + 5]) * inv_l);
@@ -1347,9 +1341,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            if (!(ok = rendezvous(bar_epi, epi_ph, kWaitEpilogue))) break;
-            if (row == 0) {
-              tma_store_4d(&map_o, stage, hh * 64, head_t, q_row0_t, item_bin);
+            __syncwarp();
+            if (lane == 0 && row0_w < args.capacity) {
+              tma_store_4d(&map_o, stage, hh * 64, head_t, row0_w, item_bin);
               asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
           }
@@ -1361,7 +1355,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       PROF_LAP(7);
       ++it_n;
     }
-    if (h == 0 && row == 0) tma_store_wait_read();     // staging must outlive the last store's read
+    if (h == 0 && lane == 0) tma_store_wait_read();    // staging must outlive the last store's read
 #ifdef PP_PROFILE
     prof_acc[10] = tcount;
     if (row == 0 && h == 0) PROF_STORE(8 + 12 * t, 12);
@@ -1467,7 +1461,7 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   if ((st = make_map(&mq, q, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
   if ((st = make_map(&mk, k, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
   if ((st = make_map(&mv, v, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
-  if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
+  if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, 32)) != PP_OK) return st;   // one warp's rows per store
   static bool configured = false;   // per process, per template instance
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<D, kIndep>, cudaFuncAttributeMaxDynamicSharedMemorySize,
