@@ -384,6 +384,16 @@ int host_pipe(HostPipe** out) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return note_cuda_error((int)e, "cudaGetDevice");
   if (pipe.device != dev) {
+    // first use on this device (or a call that failed half-way): drop whatever an earlier device or
+    // attempt left behind. Handles are destroyed with the device they were made on current.
+    if (pipe.device >= 0 && cudaSetDevice(pipe.device) != cudaSuccess) (void)cudaGetLastError();
+    for (int g = 0; g < kHostGroups; ++g) {
+      if (pipe.stream[g]) { cudaStreamDestroy(pipe.stream[g]); pipe.stream[g] = nullptr; }
+      if (pipe.done[g]) { cudaEventDestroy(pipe.done[g]); pipe.done[g] = nullptr; }
+    }
+    if (pipe.start) { cudaEventDestroy(pipe.start); pipe.start = nullptr; }
+    if (pipe.device >= 0 && (e = cudaSetDevice(dev)) != cudaSuccess) return note_cuda_error((int)e, "cudaSetDevice");
+    pipe.device = -1;
     for (int g = 0; g < kHostGroups; ++g) {
       if ((e = cudaStreamCreateWithFlags(&pipe.stream[g], cudaStreamNonBlocking)) != cudaSuccess)
         return note_cuda_error((int)e, "cudaStreamCreate");
@@ -445,6 +455,15 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
     // one group overlap the kernels of another and the downloads of a third (PCIe is full duplex).
     pp::HostPipe* pipe = nullptr;
     if ((st = pp::host_pipe(&pipe)) != PP_OK) return st;
+    // On an error in the middle of the pipeline, work already queued on the internal streams still
+    // reads and writes the caller's buffers: wait for it before handing the error back.
+    auto bail = [&](int code) {
+      for (int g = 0; g < pp::kHostGroups; ++g) (void)cudaStreamSynchronize(pipe->stream[g]);
+      (void)cudaStreamSynchronize(s);
+      return code;
+    };
+#undef PP_TRY
+#define PP_TRY(call, what) do { e = (call); if (e != cudaSuccess) return bail(pp::note_cuda_error((int)e, what)); } while (0)
     const int n_groups = (int)h.groups.size();
     PP_TRY(cudaMemsetAsync(base + h.status, 0, 4, s), "memset status");
     PP_TRY(cudaEventRecord(pipe->start, s), "event record");
@@ -466,7 +485,7 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
       const size_t attn_tab = (sizeof(int32_t) * pp::prefill_table_ints(G.n_bins, cap, kg) + 255) & ~size_t(255);
       const size_t unpack_tab = (pp::unpack_table_bytes(kg) + 255) & ~size_t(255);
       void* stage = nullptr;
-      if ((st = pp::host_staging(pipe, g, map_bytes + attn_tab + unpack_tab, &stage)) != PP_OK) return st;
+      if ((st = pp::host_staging(pipe, g, map_bytes + attn_tab + unpack_tab, &stage)) != PP_OK) return bail(st);
       int64_t* map = static_cast<int64_t*>(stage);
       g_cache_off.resize(kg);
       int64_t t = 0;
@@ -489,11 +508,11 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
       st = pp_prefill_attention(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), kg, gq, gk, gv, go,
                                 base + h.ws_attn + g * h.ws_attn_stride, static_cast<char*>(stage) + map_bytes, attn_tab,
                                 reinterpret_cast<int32_t*>(base + h.status), sg);
-      if (st != PP_OK) return st;
+      if (st != PP_OK) return bail(st);
       st = pp_unpack_kv(&gp, G.bin_of.data(), G.off_of.data(), lengths + G.i0, kg, gk, gv, base + h.kc, base + h.vc,
                         g_cache_off.data(), lengths + G.i0, base + h.ws_unpack + g * h.ws_unpack_stride,
                         static_cast<char*>(stage) + map_bytes + attn_tab, unpack_tab, sg);
-      if (st != PP_OK) return st;
+      if (st != PP_OK) return bail(st);
       gp.flags = pp::kFlagTablesReady;
       PP_TRY(cudaMemcpyAsync(base + h.q_tok + tok0 * q_row, (const char*)q_host + tok0 * q_row, ntok * q_row,
                              cudaMemcpyHostToDevice, sg), "H2D q");
@@ -507,20 +526,20 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
       PP_TRY(cudaMemsetAsync(base + h.k + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed k");
       PP_TRY(cudaMemsetAsync(base + h.v + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed v");
       mark(sg);   // memsets
-      if ((st = pp::launch_tensorize(true, gq, base + h.q_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return st;
-      if ((st = pp::launch_tensorize(true, gk, base + h.k_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return st;
-      if ((st = pp::launch_tensorize(true, gv, base + h.v_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return st;
+      if ((st = pp::launch_tensorize(true, gq, base + h.q_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return bail(st);
+      if ((st = pp::launch_tensorize(true, gk, base + h.k_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return bail(st);
+      if ((st = pp::launch_tensorize(true, gv, base + h.v_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return bail(st);
       mark(sg);   // scatter
       st = pp_prefill_attention(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), kg, gq, gk, gv, go,
                                 base + h.ws_attn + g * h.ws_attn_stride, static_cast<char*>(stage) + map_bytes, attn_tab,
                                 reinterpret_cast<int32_t*>(base + h.status), sg);
-      if (st != PP_OK) return st;
+      if (st != PP_OK) return bail(st);
       mark(sg);   // attention
       st = pp_unpack_kv(&gp, G.bin_of.data(), G.off_of.data(), lengths + G.i0, kg, gk, gv, base + h.kc, base + h.vc,
                         g_cache_off.data(), lengths + G.i0, base + h.ws_unpack + g * h.ws_unpack_stride,
                         static_cast<char*>(stage) + map_bytes + attn_tab, unpack_tab, sg);
-      if (st != PP_OK) return st;
-      if ((st = pp::launch_tensorize(false, go, base + h.o_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return st;
+      if (st != PP_OK) return bail(st);
+      if ((st = pp::launch_tensorize(false, go, base + h.o_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return bail(st);
       mark(sg);
       PP_TRY(cudaMemcpyAsync((char*)o_host + tok0 * q_row, base + h.o_tok + tok0 * q_row, ntok * q_row,
                              cudaMemcpyDeviceToHost, sg), "D2H o");
