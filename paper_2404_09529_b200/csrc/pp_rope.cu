@@ -144,10 +144,13 @@ struct SegExt {                    // per-segment arrays appended to the prefill
   int32_t off_true_len, off_cap, off_cache_off;   // int32 offsets into the table (cache_off: int64 data)
 };
 
-constexpr int kRuRows = 8;   // packed rows per block of the fused K/V kernel
+// Packed rows per block of the fused K/V kernel: 8 where a row of K is several KB (many KV heads), 32
+// where it is at most 2 KB, so that a block always has tens of KB to move for its set-up cost.
+constexpr int kRuRowsWide = 8, kRuRowsNarrow = 32;
+constexpr int kRuNarrowRowElems = 1024;   // n_kv_heads * D up to which a row counts as narrow
 constexpr int kRuV = 8;      // 16-byte V copies in flight per thread
 constexpr int kRuK = 2;      // (lower, upper) K pairs in flight per thread
-template <int D>
+template <int D, int kRuRows>
 __global__ void __launch_bounds__(kRopeThreads)
 rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
                    __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
@@ -290,18 +293,21 @@ int launch_rope_unpack(const pp_attn_params& p, const int32_t* d_table, const Ta
                        int32_t off_true_len, int32_t off_cap, int32_t off_cache_off, const void* rope_table,
                        void* k, const void* v, void* k_cache, void* v_cache, void* stream) {
   const int64_t n_rows = (int64_t)p.n_bins * p.capacity;
-  const unsigned grid = (unsigned)((n_rows + kRuRows - 1) / kRuRows);
+  const bool narrow = p.n_kv_heads * p.head_dim <= kRuNarrowRowElems;
+  const int rows = narrow ? kRuRowsNarrow : kRuRowsWide;
+  const unsigned grid = (unsigned)((n_rows + rows - 1) / rows);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const SegExt ext{off_true_len, off_cap, off_cache_off};
+#define PP_RU_LAUNCH(DD, RR)                                                                                      \
+  rope_unpack_kernel<DD, RR><<<grid, kRopeThreads, 0, s>>>(                                                       \
+      (__nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table,      \
+      L.bin_seg_ptr, L.bin_used, L.seg_start, ext, (const float2*)rope_table, p.n_bins, p.capacity, p.n_kv_heads)
   if (p.head_dim == 128) {
-    rope_unpack_kernel<128><<<grid, kRopeThreads, 0, s>>>(
-        (__nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table,
-        L.bin_seg_ptr, L.bin_used, L.seg_start, ext, (const float2*)rope_table, p.n_bins, p.capacity, p.n_kv_heads);
+    if (narrow) PP_RU_LAUNCH(128, kRuRowsNarrow); else PP_RU_LAUNCH(128, kRuRowsWide);
   } else {
-    rope_unpack_kernel<64><<<grid, kRopeThreads, 0, s>>>(
-        (__nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table,
-        L.bin_seg_ptr, L.bin_used, L.seg_start, ext, (const float2*)rope_table, p.n_bins, p.capacity, p.n_kv_heads);
+    if (narrow) PP_RU_LAUNCH(64, kRuRowsNarrow); else PP_RU_LAUNCH(64, kRuRowsWide);
   }
+#undef PP_RU_LAUNCH
   const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "rope+unpack kernel launch");
 }
