@@ -551,40 +551,66 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           PROF_LAP(3);
           return true;
         };
-        while (ok) {
-          const uint32_t ring = it_n % kRing;
-          if (!mbar_wait(b_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull)) break;
-          const volatile int* e = s_ring + (t * (int)kRing + (int)ring) * kRingInts;
-          const int w = e[0], n = e[3];
-          mbar_arrive(b_item_empty + 8 * ring);
-          if (w < 0) break;
-          PROF_LAP(0);
-          if (!(ok = mbar_wait(bar_q_ready, it_n & 1u, wctx, kWaitQFull))) break;
-          PROF_LAP(1);
-          if (!(ok = issue_qk(kc, n == 1))) break;
-          for (int j = 0; j < n; ++j, ++kc) {
-            if (j + 1 < n && !(ok = issue_qk(kc + 1, j + 2 == n))) break;
-            // the previous item's epilogue must have read O_t before it is overwritten
-            if (j == 0 && !(ok = mbar_wait(b_o_empty, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
-            PROF_LAP(4);
-            const uint32_t b = kc & 1u, parity = (kc >> 1) & 1u;
-            if (!(ok = mbar_wait(b_p_full + 8 * b, parity, wctx, kWaitP))) break;
-            PROF_LAP(5);
-            if (!(ok = mbar_wait(b_v_full + 8 * b, parity, wctx, kWaitVFull))) break;
-            PROF_LAP(6);
-            tc_fence_after();            // O_t (+)= P(k) V(k)
-            const uint32_t a = tm_s + 64u * b;
-            const uint32_t vb = v_lo + b * (Cfg::kKVBytes >> 4);
-            mma_ts(tm_o, a, vb, idesc_pv, j == 0 ? 0u : 1u);
-#pragma unroll
-            for (int kk = 1; kk < BN / 16; ++kk)
-              mma_ts(tm_o, a + kk * 8, vb + (uint32_t)kk * ((16 * 128) >> 4), idesc_pv, 1u);
-            tc_commit(b_v_empty + 8 * b);
-            PROF_LAP(7);
+        // The slot's tiles form one stream across items: while the softmax threads work on tile k,
+        // the scores of the stream's next tile are computed, also when that tile opens the slot's
+        // next item (its Q was loaded as soon as this item's last scores had been issued).
+        int w = -1, n = 0, j = 0;
+        {
+          if (!mbar_wait(b_item_full, 0u, wctx, kWaitItemFull)) ok = false;
+          if (ok) {
+            const volatile int* e = s_ring + (t * (int)kRing) * kRingInts;
+            w = e[0]; n = e[3];
+            mbar_arrive(b_item_empty);
           }
-          if (!ok) break;
-          tc_commit(b_o_full);
-          ++it_n;
+        }
+        PROF_LAP(0);
+        if (ok && w >= 0) ok = mbar_wait(bar_q_ready, 0u, wctx, kWaitQFull) && issue_qk(kc, n == 1);
+        while (ok && w >= 0) {
+          const bool last_tile = (j + 1 == n);
+          int w_next = w, n_next = n;
+          bool have = true, last_flag = (j + 2 == n);
+          // With one tile per item the next item's scores would be issued before the previous item's
+          // epilogue has read O_t; the softmax threads must not get that far ahead of it.
+          if (j == 0 && last_tile && !(ok = mbar_wait(b_o_empty, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
+          if (last_tile) {
+            const uint32_t item = it_n + 1u, ring = item % kRing;
+            PROF_LAP(4);
+            if (!(ok = mbar_wait(b_item_full + 8 * ring, (item / kRing) & 1u, wctx, kWaitItemFull))) break;
+            const volatile int* e = s_ring + (t * (int)kRing + (int)ring) * kRingInts;
+            w_next = e[0]; n_next = e[3];
+            mbar_arrive(b_item_empty + 8 * ring);
+            PROF_LAP(0);
+            have = w_next >= 0;
+            last_flag = n_next == 1;
+            if (have && !(ok = mbar_wait(bar_q_ready, item & 1u, wctx, kWaitQFull))) break;
+            PROF_LAP(1);
+          }
+          if (have && !(ok = issue_qk(kc + 1, last_flag))) break;
+          // the previous item's epilogue must have read O_t before it is overwritten
+          if (j == 0 && !last_tile && !(ok = mbar_wait(b_o_empty, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
+          PROF_LAP(4);
+          const uint32_t b = kc & 1u, parity = (kc >> 1) & 1u;
+          if (!(ok = mbar_wait(b_p_full + 8 * b, parity, wctx, kWaitP))) break;
+          PROF_LAP(5);
+          if (!(ok = mbar_wait(b_v_full + 8 * b, parity, wctx, kWaitVFull))) break;
+          PROF_LAP(6);
+          tc_fence_after();            // O_t (+)= P(k) V(k)
+          const uint32_t a = tm_s + 64u * b;
+          const uint32_t vb = v_lo + b * (Cfg::kKVBytes >> 4);
+          mma_ts(tm_o, a, vb, idesc_pv, j == 0 ? 0u : 1u);
+#pragma unroll
+          for (int kk = 1; kk < BN / 16; ++kk)
+            mma_ts(tm_o, a + kk * 8, vb + (uint32_t)kk * ((16 * 128) >> 4), idesc_pv, 1u);
+          tc_commit(b_v_empty + 8 * b);
+          PROF_LAP(7);
+          ++kc;
+          if (last_tile) {
+            tc_commit(b_o_full);
+            ++it_n;
+            w = w_next; n = n_next; j = 0;
+          } else {
+            ++j;
+          }
         }
         if (t == 0) PROF_STORE(0, 8);
       }
