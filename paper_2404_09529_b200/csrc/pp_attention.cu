@@ -841,12 +841,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const int kv0 = item_kv_row0 + j * BN;
             const int c_lo = max(key_lo - kv0, 0);
             const int c_hi = min(key_hi - kv0, EPT - 1);         // visible columns [c_lo, c_hi]
-            const bool full = (c_lo == 0) && (c_hi == EPT - 1);
-            const bool warp_full = __all_sync(0xffffffffu, full);
-            bool need[NCH];
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch)
-              need[ch] = __any_sync(0xffffffffu, max(c_lo, 32 * ch) <= min(c_hi, 32 * ch + 31));
+            // one warp reduction for all the per-warp flags of the tile: which 32-column chunks
+            // somebody can see, and whether any row's interval ends or begins inside the tile
+            static_assert(NCH == 2, "flag bits below are laid out for two chunks");
+            const uint32_t lane_flags = (uint32_t)(c_lo <= min(c_hi, 31)) | ((uint32_t)(max(c_lo, 32) <= c_hi) << 1) |
+                                        ((uint32_t)(c_hi < EPT - 1) << 2) | ((uint32_t)(c_lo > 0) << 3);
+            const uint32_t warp_flags = __reduce_or_sync(0xffffffffu, lane_flags);
+            const bool need[NCH] = {(warp_flags & 1u) != 0, (warp_flags & 2u) != 0};
+            const bool cut_hi = (warp_flags & 4u) != 0, cut_lo = (warp_flags & 8u) != 0;
             const uint32_t sbuf = tcount & 1u;                   // tile k of the stream lives in S buffer k & 1
             const uint32_t tmem_sb = tmem_s + 64u * sbuf;
             PROF_LAP(5);
@@ -866,15 +868,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             tc_wait_ld();
             PROF_LAP(2);
-            if (!warp_full) {
-              if (__any_sync(0xffffffffu, c_hi < EPT - 1)) {
+            // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
+            // one of the two bounds (the causal diagonal, or the first tile of a prompt)
+            if (cut_hi) {
 #pragma unroll
-                for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
-              }
-              if (__any_sync(0xffffffffu, c_lo > 0)) {
+              for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
+            }
+            if (cut_lo) {
 #pragma unroll
-                for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
-              }
+              for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
             }
             float mx;
             {
