@@ -1152,8 +1152,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     };
     while (true) {
       // in independent mode slot t has its own ring, and an item describes one tile (its slot-0 fields)
-      const uint32_t ring = (kIndep ? (uint32_t)t * kRing : 0u) + it_n % kRing;
-      const int f = kIndep ? 0 : t;                    // which slot fields of the entry to read
+      const uint32_t ring = it_n % kRing;
+      const int f = t;                                 // which slot fields of the entry to read
       PROF_LAP(8);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull));
       PROF_LAP(0);
@@ -1192,16 +1192,17 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int kv0 = item_kv_row0 + j * BN + EPT * h;     // first key of this thread's half
         const int c_lo = max(key_lo - kv0, 0);
         const int c_hi = min(key_hi - kv0, EPT - 1);         // visible columns [c_lo, c_hi] of the half
-        const bool full = (c_lo == 0) && (c_hi == EPT - 1);
-        const bool warp_full = __all_sync(0xffffffffu, full);
-        bool need[NCH];
-#pragma unroll
-        for (int ch = 0; ch < NCH; ++ch)
-          need[ch] = __any_sync(0xffffffffu, max(c_lo, 32 * ch) <= min(c_hi, 32 * ch + 31));
-        // independent mode: tile k of the slot's stream lives in S buffer k & 1
-        const uint32_t sbuf = kIndep ? (tcount & 1u) : 0u;
-        const uint32_t tparity = kIndep ? ((tcount >> 1) & 1u) : (tcount & 1u);
-        const uint32_t tmem_sb = tmem_s + 64u * sbuf;
+        // one warp reduction for all the per-warp flags of the tile: which 32-column chunks somebody
+        // can see, and whether any row's interval ends or begins inside this half of the tile
+        static_assert(NCH == 2, "flag bits below are laid out for two chunks");
+        const uint32_t lane_flags = (uint32_t)(c_lo <= min(c_hi, 31)) | ((uint32_t)(max(c_lo, 32) <= c_hi) << 1) |
+                                    ((uint32_t)(c_hi < EPT - 1) << 2) | ((uint32_t)(c_lo > 0) << 3);
+        const uint32_t warp_flags = __reduce_or_sync(0xffffffffu, lane_flags);
+        const bool need[NCH] = {(warp_flags & 1u) != 0, (warp_flags & 2u) != 0};
+        const bool cut_hi = (warp_flags & 4u) != 0, cut_lo = (warp_flags & 8u) != 0;
+        const uint32_t sbuf = 0u;
+        const uint32_t tparity = tcount & 1u;
+        const uint32_t tmem_sb = tmem_s;
         PROF_LAP(5);
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * (2 * t + sbuf), tparity, wctx, kWaitS));
         if (!ok) break;                                      // warp-uniform
@@ -1221,17 +1222,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         tc_wait_ld();
         PROF_LAP(2);
-        if (!warp_full) {
-          // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
-          // one of the two bounds (the causal diagonal, or the first tile of a prompt)
-          if (__any_sync(0xffffffffu, c_hi < EPT - 1)) {
+        // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
+        // one of the two bounds (the causal diagonal, or the first tile of a prompt)
+        if (cut_hi) {
 #pragma unroll
-            for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
-          }
-          if (__any_sync(0xffffffffu, c_lo > 0)) {
+          for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
+        }
+        if (cut_lo) {
 #pragma unroll
-            for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
-          }
+          for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
         }
         float mx;
         {
@@ -1264,16 +1263,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const bool rescale = (m_new != m_run) && (m_run != -INFINITY);
         const float alpha = rescale ? fast_exp2(m_run - m_new) : 1.f;
         if (j > jb_t && __any_sync(0xffffffffu, rescale)) {
-          if constexpr (kIndep) {
-            // S(k) is computed ahead of P(k-1) V(k-1) here, so O_t is stable only once that product
-            // has been committed: the release of the V stage it read is the same event
-            const uint32_t kp = tcount - 1u;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_v_empty + 8 * (2 * t + (kp & 1u)), (kp >> 1) & 1u, wctx, kWaitVEmpty));
-            if (!ok) break;
-            tc_fence_after();
-          }
-          // (shared mode: S_t ready implies the previous P_t V product has finished.) Each half
-          // rescales its own D/2 columns of the row.
+          // (S_t ready implies that the previous P_t V product has finished.) Each half rescales its
+          // own D/2 columns of the row.
 #pragma unroll 1
           for (int ch = 0; ch < D / 32; ++ch) {          // rare path: keep it small
             uint32_t ov[16];
