@@ -34,7 +34,7 @@ DEFAULT_WORKLOAD = "llama2_7b"
 # DRAM traffic of one attention-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu capture summarised in profiles/attention_llama2_7b.md; None where no capture exists for
 # the workload.
-NCU_ATTENTION_TRAFFIC_BYTES = {"llama2_7b": 563.2e6}
+NCU_ATTENTION_TRAFFIC_BYTES = {"llama2_7b": 562.2e6}
 
 
 def load_peaks():
