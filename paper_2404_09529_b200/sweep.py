@@ -45,6 +45,11 @@ def _time_ms(fn, iters: int = 5, warmup: int = 2) -> float:
         fn()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # a few milliseconds of device-side delay first, so that the host has queued every call before
+    # the first one starts: the events then bracket device time, not the host's enqueue rate (these
+    # batches are small enough for a step to be shorter than the time it takes to enqueue it)
+    if hasattr(torch.cuda, "_sleep"):
+        torch.cuda._sleep(4_000_000)
     e0.record()
     for _ in range(iters):
         fn()
