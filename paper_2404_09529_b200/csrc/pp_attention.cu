@@ -452,6 +452,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem_base;
+  // Everything above is set-up that touches no tensor: with a programmatic dependent launch it runs
+  // while the kernel before this one (rotation / cache scatter) is still finishing.
+  pdl_wait();
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
@@ -1513,8 +1516,9 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   a.status = device_status;
   a.wait_limit_ns = wait_limit_ns();
   const unsigned grid = (unsigned)(total < sms ? total : sms);
-  attention_kernel<D, kIndep><<<grid, kAttnThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, mo, a);
-  const cudaError_t e = cudaGetLastError();
+  const cudaError_t launch_err = launch_dependent(attention_kernel<D, kIndep>, dim3(grid), dim3(kAttnThreads),
+                                                  (size_t)Cfg::kSmemBytes, stream, mq, mk, mv, mo, a);
+  const cudaError_t e = launch_err != cudaSuccess ? launch_err : cudaGetLastError();
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "attention kernel launch");
 }
 

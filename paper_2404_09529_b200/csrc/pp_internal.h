@@ -86,6 +86,33 @@ int launch_bounded_wait_selftest(int32_t* device_status, uint64_t limit_ns, void
 // cache_cap[k], cache_off as int64[k] (8-byte aligned).
 size_t unpack_table_bytes(int32_t k);
 
+#ifdef __CUDACC__
+// Programmatic dependent launch. A kernel of the path that is launched with launch_dependent() may
+// start while the kernel before it in the stream is still finishing: its blocks are scheduled once
+// every block of that kernel has called pdl_launch_dependents() (or exited), run their set-up, and
+// block in pdl_wait() until that kernel has completed and its writes are visible. Work queued
+// before that kernel has completed by then in any case. Launched the ordinary way, both calls
+// do nothing.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif  // __CUDACC__
+
 }  // namespace pp
 
 #endif  // PREPACK_B200_PP_INTERNAL_H_

@@ -53,6 +53,7 @@ rope_kernel(const __nv_bfloat16* q, __nv_bfloat16* q_out, __nv_bfloat16* __restr
   __shared__ float s_cos[kRopeRows][kHalf];
   __shared__ float s_sin[kRopeRows][kHalf];
 
+  pdl_launch_dependents();      // the attention kernel may set up while this one runs
   const int64_t row0 = (int64_t)blockIdx.x * kRopeRows;
   const int64_t n_rows = (int64_t)n_bins * capacity;
   const int tid = threadIdx.x;
@@ -123,6 +124,7 @@ rope_kernel(const __nv_bfloat16* q, __nv_bfloat16* q_out, __nv_bfloat16* __restr
 __global__ void __launch_bounds__(256)
 rope_table_kernel(float2* __restrict__ table, int32_t capacity, int32_t half,
                   const __grid_constant__ RopeFreq freq) {
+  pdl_launch_dependents();      // the fused K/V kernel may set up while this one runs
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)capacity * half) return;
   const int32_t pos = (int32_t)(idx / half), j = (int32_t)(idx - (int64_t)pos * half);
@@ -165,6 +167,7 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
   __shared__ int64_t s_head_stride[kRuRows];      // cache_cap * D
   __shared__ float4 s_tab[kRuRows][D / 4];          // (cos, sin) of j = 2g, 2g + 1 at each row's position
 
+  pdl_launch_dependents();      // the attention kernel may set up while this one runs
   const int64_t row0 = (int64_t)blockIdx.x * kRuRows;
   const int64_t n_rows = (int64_t)n_bins * capacity;
   const int tid = threadIdx.x;
@@ -194,6 +197,7 @@ rope_unpack_kernel(__nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     s_head_stride[tid] = stride;
   }
   __syncthreads();
+  pdl_wait();                   // the rotation table is written by the kernel before this one
   // each row's D/2 (cos, sin) pairs once, for all heads: D/4 16-byte loads per row, one per thread
   for (int u = tid; u < kRuRows * (D / 4); u += kRopeThreads) {
     const int r = u / (D / 4), g = u - r * (D / 4);
@@ -298,8 +302,9 @@ int launch_rope_unpack(const pp_attn_params& p, const int32_t* d_table, const Ta
   const unsigned grid = (unsigned)((n_rows + rows - 1) / rows);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const SegExt ext{off_true_len, off_cap, off_cache_off};
+  cudaError_t launch_err = cudaSuccess;
 #define PP_RU_LAUNCH(DD, RR)                                                                                      \
-  rope_unpack_kernel<DD, RR><<<grid, kRopeThreads, 0, s>>>(                                                       \
+  launch_err = launch_dependent(rope_unpack_kernel<DD, RR>, dim3(grid), dim3(kRopeThreads), 0, s,                 \
       (__nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table,      \
       L.bin_seg_ptr, L.bin_used, L.seg_start, ext, (const float2*)rope_table, p.n_bins, p.capacity, p.n_kv_heads)
   if (p.head_dim == 128) {
@@ -308,7 +313,7 @@ int launch_rope_unpack(const pp_attn_params& p, const int32_t* d_table, const Ta
     if (narrow) PP_RU_LAUNCH(64, kRuRowsNarrow); else PP_RU_LAUNCH(64, kRuRowsWide);
   }
 #undef PP_RU_LAUNCH
-  const cudaError_t e = cudaGetLastError();
+  const cudaError_t e = launch_err != cudaSuccess ? launch_err : cudaGetLastError();
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "rope+unpack kernel launch");
 }
 
