@@ -39,6 +39,7 @@ decode_append_kernel(const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat1
                      const __grid_constant__ DecodeFreq freq) {
   constexpr int kHalf = D / 2;
   __shared__ float s_cos[kHalf], s_sin[kHalf];
+  pdl_launch_dependents();      // the partial kernel may set up while this one runs
   const int i = blockIdx.x;
   const int32_t pos = table[T.lengths + i];                      // position of the new token
   const int64_t cap = table[T.cache_cap + i];
@@ -125,6 +126,8 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q_rot, const __nv_bfloat
   const int i = table[T.chunks + 3 * chunk], key0 = table[T.chunks + 3 * chunk + 1], n_keys = table[T.chunks + 3 * chunk + 2];
   const int64_t cap = table[T.cache_cap + i];
   const int64_t base = reinterpret_cast<const int64_t*>(table + T.cache_off)[i] + (int64_t)kvh * cap * D;
+  pdl_launch_dependents();      // the combine kernel may set up while this one runs
+  pdl_wait();                   // rotated queries and the appended K / V rows come from the append kernel
   float q[G][E], acc[G][E], m[G], l[G];
 #pragma unroll
   for (int h = 0; h < G; ++h) {
@@ -217,6 +220,7 @@ decode_combine_kernel(const float* __restrict__ partial, __nv_bfloat16* __restri
                       const int32_t* __restrict__ table, DecodeTable T, int32_t n_q_heads) {
   const int i = blockIdx.x, head = blockIdx.y, d = threadIdx.x;
   const int c0 = table[T.chunk_ptr + i], c1 = table[T.chunk_ptr + i + 1];
+  pdl_wait();                   // the partial results come from the kernel before this one
   float mm = -INFINITY;
   for (int c = c0; c < c1; ++c) mm = fmaxf(mm, partial[((int64_t)c * n_q_heads + head) * (D + 2)]);
   float ll = 0.f, oo = 0.f;
@@ -340,9 +344,10 @@ extern "C" int pp_decode_step(const pp_attn_params* params, const int32_t* lengt
   const float scale_log2 = scale * 1.4426950408889634f;
   const int group = params->n_q_heads / params->n_kv_heads;
   const dim3 grid_p((unsigned)L.n_chunks, (unsigned)params->n_kv_heads), grid_c((unsigned)k, (unsigned)params->n_q_heads);
+  cudaError_t le = cudaSuccess;
 #define PP_DECODE_PARTIAL(DD, GG)                                                                                \
-  pp::decode_partial_kernel<DD, GG><<<grid_p, pp::kDecodeThreads, 0, s>>>(                                       \
-      q_rot, (const __nv_bfloat16*)k_cache, (const __nv_bfloat16*)v_cache, partial, d_table, L.T,                \
+  le = pp::launch_dependent(pp::decode_partial_kernel<DD, GG>, grid_p, dim3(pp::kDecodeThreads), 0, s,           \
+      (const __nv_bfloat16*)q_rot, (const __nv_bfloat16*)k_cache, (const __nv_bfloat16*)v_cache, partial, d_table, L.T, \
       params->n_q_heads, params->n_kv_heads, group, scale_log2)
 #define PP_DECODE_LAUNCH(DD)                                                                                     \
   pp::decode_append_kernel<DD><<<k, pp::kDecodeThreads, 0, s>>>(                                                 \
@@ -350,10 +355,12 @@ extern "C" int pp_decode_step(const pp_attn_params* params, const int32_t* lengt
       (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, d_table, L.T, params->n_q_heads, params->n_kv_heads, freq); \
   if (group == 1) PP_DECODE_PARTIAL(DD, 1); else if (group == 2) PP_DECODE_PARTIAL(DD, 2);                       \
   else if (group <= 4) PP_DECODE_PARTIAL(DD, 4); else PP_DECODE_PARTIAL(DD, 8);                                  \
-  pp::decode_combine_kernel<DD><<<grid_c, DD, 0, s>>>(partial, (__nv_bfloat16*)o, d_table, L.T, params->n_q_heads)
+  if (le == cudaSuccess)                                                                                         \
+    le = pp::launch_dependent(pp::decode_combine_kernel<DD>, grid_c, dim3(DD), 0, s, (const float*)partial,      \
+                              (__nv_bfloat16*)o, d_table, L.T, params->n_q_heads)
   if (params->head_dim == 128) { PP_DECODE_LAUNCH(128); } else { PP_DECODE_LAUNCH(64); }
 #undef PP_DECODE_LAUNCH
 #undef PP_DECODE_PARTIAL
-  e = cudaGetLastError();
+  e = le != cudaSuccess ? le : cudaGetLastError();
   return e == cudaSuccess ? PP_OK : pp::note_cuda_error((int)e, "decode kernel launch");
 }
