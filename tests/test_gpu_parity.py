@@ -91,6 +91,8 @@ def test_large_configs_sampled_parity_packed(name):
     ([700, 300, 250, 150, 90, 5, 5], 8, 2, 128),   # several tiles, segments straddling tiles
     ([515, 130, 129, 128, 64, 33, 17, 9, 3, 2, 1], 8, 1, 64),   # group 8, D = 64
     ([8] * 40, 2, 2, 64),                  # many equal short prompts: 16 segments per tile
+    ([300] + [1, 2, 3, 1, 2] * 60, 4, 4, 64),      # one- to three-token prompts: > 32 prompt starts in a tile
+    ([4096, 4096] + [2] * 700 + [1] * 300, 4, 2, 128),   # the same next to long prompts (shared-stream mode)
 ])
 def test_edge_shapes_full_parity(lengths, hq, hkv, d):
     q, k, v = _random_case(lengths, hq, hkv, d, seed=len(lengths) * 1000 + d)
