@@ -129,7 +129,12 @@ size_t pp_prefill_workspace_bytes(const pp_attn_params* params, int32_t k);
  *                   builds the tables here and copies them with one async H2D on `stream`; it
  *                   must stay untouched until that copy has run
  *   device_status   device int32 or NULL; set non-zero by the kernel if a bounded wait inside
- *                   it gave up (then outputs are invalid). The caller zeroes and reads it.
+ *                   it gave up (then outputs are invalid). The caller zeroes and reads it. Every
+ *                   wait in the kernel is limited to 2 s; the environment variables
+ *                   PP_WAIT_LIMIT_MS / PP_WAIT_LIMIT_US, read at each call, override the limit.
+ * The kernels of one call may be launched as programmatic dependents of one another (set-up of a
+ * kernel overlapping the end of the kernel before it); nothing of that is visible to the caller:
+ * stream order holds for everything the caller enqueues before and after the call.
  * Arithmetic: rotation in fp32 with one rounding to bf16; scores and outputs accumulated in
  * fp32 on the tensor cores, probabilities rounded to bf16 before the P.V product.
  * Errors (all detected before anything is enqueued): PP_ERR_INVALID_ARG, PP_ERR_LENGTH,
