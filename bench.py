@@ -190,21 +190,48 @@ def oracle_sample(cfg, lengths, budget_s, max_prompts=None):
     return tokens, time.perf_counter() - t0, done
 
 
+def workload_config(cfg, name, lengths, n_bins, capacity, world):
+    """The `config` object of the JSON line; both arms (--impl ours / reference) print the same one."""
+    d, hq, hkv = cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads
+    T = int(lengths.sum())
+    rows = int(n_bins) * int(capacity)
+    # one step touches q, k (read and written back), v, o and both cache pools
+    stream_mb = (rows * d * 2 * (2 * hq + 3 * hkv) + T * d * 2 * 2 * hkv) / 1e6
+    l2 = (f"no flush: each step streams {stream_mb:.0f} MB of tensors, larger than the 126 MB L2"
+          if stream_mb > 2 * 126 else
+          f"flushed: each step touches only {stream_mb:.1f} MB, so a 256 MB buffer is overwritten before every "
+          "timed step and the steps are timed one by one")
+    return {"workload": name, "description": cfg.description, "n_prompts": int(len(lengths)),
+            "total_tokens": T, "n_bins": int(n_bins), "capacity": int(capacity),
+            "n_q_heads": hq, "n_kv_heads": hkv, "head_dim": d, "rope_base": cfg.rope_base, "path": "fused",
+            "parallelism": f"replicas x{world}" if world > 1 else "single GPU", "l2": l2}, stream_mb
+
+
 def run_reference(args):
-    """--impl reference: the float64 CPU oracle on the host cores, bounded sample per step."""
+    """--impl reference: the float64 CPU oracle on the host cores. Every step is the whole workload
+    where `--steps + --warmup` such passes fit in about five minutes, otherwise a bounded sample of it
+    (the first prompts in original order), named in cpu_baseline.sample."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    from oracle import prepack_oracle as orc
     from workloads import CONFIGS, prompt_lengths
     cfg = CONFIGS[args.workload]
     lengths = prompt_lengths(args.workload)
     cores = len(os.sched_getaffinity(0))
-    # size the per-step sample from one calibration run so that the whole run stays within minutes
     total_steps = args.steps + args.warmup
-    per_step_budget = max(0.5, min(8.0, 120.0 / max(total_steps, 1)))
-    tok, sec, n_cal = oracle_sample(cfg, lengths, per_step_budget)
-    n_prompts = n_cal
-    for _ in range(max(args.warmup - 1, 0)):
+    # calibrate on a short sample: the oracle's cost per prompt grows with l^2 (attention) and l (the rest)
+    tok, sec, n_cal = oracle_sample(cfg, lengths, 2.0)
+    l = lengths.astype(np.float64)
+    work = l * l + 256.0 * l
+    est_whole = sec * work.sum() / work[:n_cal].sum()
+    if est_whole * total_steps <= 300.0:
+        n_prompts = len(lengths)
+    else:
+        per_step_budget = max(0.5, 120.0 / max(total_steps, 1))
+        cum = np.cumsum(work) * (sec / work[:n_cal].sum())
+        n_prompts = max(1, int(np.searchsorted(cum, per_step_budget, side="right")))
+    for _ in range(args.warmup):
         oracle_sample(cfg, lengths, 1e9, n_prompts)
     t_tot, tok_tot = 0.0, 0
     for _ in range(args.steps):
@@ -212,12 +239,16 @@ def run_reference(args):
         t_tot += sec
         tok_tot += tok
     value = tok_tot / t_tot
-    sample = f"first {n_prompts} of {len(lengths)} prompts ({tok} tokens) per step, all heads, numpy float64"
+    whole = n_prompts == len(lengths)
+    sample = (f"the whole workload per step ({tok} tokens, {len(lengths)} prompts), all heads, numpy float64" if whole else
+              f"first {n_prompts} of {len(lengths)} prompts ({tok} tokens) per step, all heads, numpy float64")
+    pk = orc.ffd_pack([int(x) for x in lengths])
+    config, _ = workload_config(cfg, args.workload, lengths, pk["n_bins"], pk["capacity"], 1)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / max(args.steps, 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "description": cfg.description, "sample": sample},
+        "config": config,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -273,8 +304,12 @@ def main():
     batch.load(q_tok, k_tok, v_tok)
     # The whole path has two public routes through the C ABI: three calls (pp_pack +
     # pp_prefill_attention + pp_unpack_kv) or two (pp_pack + pp_prefill_fused). Both are timed over the
-    # same K steps; the headline is the faster one (named in config.path), the other is reported beside it.
+    # same K steps; the headline is the fused route (config.path), the other is reported beside it.
     routes = {"three_call": lambda: batch.run(repack=True), "fused": lambda: batch.run_fused(repack=True)}
+    config, stream_mb = workload_config(cfg, args.workload, lengths, batch.pack.n_bins, batch.pack.capacity, world)
+    # A step that touches less than about twice the L2 would find its inputs there on the next step:
+    # such workloads are timed step by step, with a 256 MB buffer overwritten before each.
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if stream_mb <= 2 * 126 else None
 
     def timed_region(step):
         batch.load(q_tok, k_tok, v_tok)          # raw Q/K again (the three-call route rotates q in place)
@@ -283,14 +318,24 @@ def main():
         barrier()
         sampler = ClockSampler(torch.cuda.current_device())
         sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
-        e0.record()
-        for _ in range(args.steps):
-            step()
-        e1.record()
-        barrier()
-        ms = e0.elapsed_time(e1)
+        if flush is None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                step()
+            e1.record()
+            barrier()
+            ms = e0.elapsed_time(e1)
+        else:
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+            for a, b in evs:
+                flush.fill_(1)
+                a.record()
+                step()
+                b.record()
+            barrier()
+            ms = sum(a.elapsed_time(b) for a, b in evs)
         clk = sampler.stop()
         if batch.device_status() != 0:
             raise SystemExit("device-side wait gave up during the timed region")
@@ -299,11 +344,7 @@ def main():
     route_ms, route_clocks = {}, {}
     for name, fn in routes.items():
         route_ms[name], route_clocks[name] = timed_region(fn)
-    path = min(route_ms, key=route_ms.get)
-    if dist is not None:                          # all ranks must agree on the headline route
-        flag = torch.tensor([0 if path == "three_call" else 1], device="cuda")
-        dist.broadcast(flag, src=0)
-        path = "three_call" if int(flag.item()) == 0 else "fused"
+    path = "fused"
     ms_per_step, clocks = route_ms[path], route_clocks[path]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     value = whole_job_tokens_per_s(world, T, ms_per_step)
@@ -449,17 +490,14 @@ def main():
                                   f"all heads, numpy float64, {sec:.1f} s"}
 
     if rank == 0:
-        resident_mb = (batch.q.numel() * 2 + batch.kk.numel() * 2 * 2 + batch.k_cache.numel() * 2 * 2) * 2 / 1e6
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "description": cfg.description, "n_prompts": int(len(lengths)),
-                       "total_tokens": T, "n_bins": int(batch.pack.n_bins), "capacity": int(batch.pack.capacity),
-                       "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
-                       "rope_base": cfg.rope_base, "path": path, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                       "l2": f"no flush: each step streams {resident_mb:.0f} MB of tensors, larger than the 126 MB L2"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roofline,
+            "config": config,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * args.steps, "roofline": roofline,
+            "launches_note": "fused route: rope_unpack_kernel + attention_kernel per step; the cos/sin table "
+                             "kernel runs once (first warm-up step) and is kept while the bin capacity stays the same",
             "cpu_baseline": cpu_baseline, "host": host, "kernels": kernels, "padded": padded,
             "routes": {"three_call": {"tokens_per_s": whole_job_tokens_per_s(world, T, route_ms["three_call"]),
                                       "ms_per_step": route_ms["three_call"],

@@ -46,10 +46,15 @@ enum {
   PP_ERR_TOO_LARGE = -9         /* more prompts than the built-in scratch of a *_static call   */
 };
 
-/* Flags for pp_attn_params.flags */
+/* Flags for pp_attn_params.flags. Every other bit must be zero: the entry points that read the
+ * field answer PP_ERR_INVALID_ARG to a bit they do not know. */
 enum {
   PP_FLAG_SKIP_ROPE = 1,  /* q and k already carry the rotary encoding: run attention only     */
-  PP_FLAG_ROPE_ONLY = 2   /* apply the restart rotary encoding to q and k, skip attention      */
+  PP_FLAG_ROPE_ONLY = 2,  /* apply the restart rotary encoding to q and k, skip attention      */
+  PP_FLAG_KEEP_ROPE_TABLE = 4  /* pp_prefill_fused only: the workspace was last used by a
+                             pp_prefill_fused call with the same capacity, head_dim and rope_base
+                             and nothing else has written to it since, so its cos/sin table is
+                             still valid and is not rebuilt                                      */
 };
 
 typedef struct pp_attn_params {
@@ -102,6 +107,27 @@ int pp_pack(const int32_t* lengths, int32_t k, int32_t capacity,
 int pp_fill_position_ids(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
                          const int32_t* seg_start, const int32_t* seg_len,
                          int32_t* position_ids, int32_t* segment_ids);
+
+/*
+ * How the attention kernel will walk a packed batch -- the INDEPENDENT-MASK step of Algorithm 1 and
+ * Section 3.2 turned into a tile work list: a query tile visits only the key tiles between the start
+ * of the first prompt it touches and its own last row. Host only, launches nothing; for tests, cost
+ * models and schedulers. info (int32[8], caller-allocated) receives
+ *   [0] mode: 0 = shared-stream (the two query tiles of a CTA share one stream of 128-row key
+ *       tiles; long prompts), 1 = independent (every query tile walks its own 64-row key tiles)
+ *   [1] pairing of the two query tiles of a work item: 0 = two query heads of one KV head over the
+ *       same rows, 1 = two consecutive row tiles of one head, 2 = none (independent mode)
+ *   [2] work-list entries (per KV head and head pair / head)
+ *   [3] (query tile, key tile) steps summed over the entries
+ *   [4] key rows per tile (128 or 64)
+ *   [5] entries whose second query tile is unused (the unpaired last row tile of a bin)
+ *   [6] entries whose second query tile joins the key stream after its first tile
+ *   [7] query heads folded into the rows of one query tile (1 = none)
+ * Errors: PP_ERR_INVALID_ARG, PP_ERR_LENGTH, PP_ERR_UNSUPPORTED, PP_ERR_NO_MEMORY.
+ */
+int pp_prefill_schedule_info(const pp_attn_params* params, const int32_t* bin_seg_ptr,
+                             const int32_t* seg_start, const int32_t* seg_len, int32_t k,
+                             int32_t* info);
 
 /*
  * Bytes of workspace pp_prefill_attention needs, for a batch of k prompts packed as `params`
@@ -258,9 +284,9 @@ int pp_decode_step(const pp_attn_params* params, const int32_t* lengths, int32_t
 /*
  * Whole path from host memory (Algorithm 1 (bin size to UNPACK) for one attention layer), for callers whose
  * tensors live on the host. Every tensor goes up in large contiguous copies, is laid out as the
- * packed batch by a device kernel (TENSORIZE, padding rows zeroed), pp_prefill_attention and
- * pp_unpack_kv run there, O is gathered back into token order and the outputs are copied back;
- * `stream` is synchronised before the call returns.
+ * packed batch by device kernels (TENSORIZE, padding rows zeroed), the kernels of pp_prefill_fused
+ * run there and write the caches in token order, O is gathered back into token order and the
+ * outputs are copied back; `stream` is synchronised before the call returns.
  *   params                   n_q_heads, n_kv_heads, head_dim, rope_base, softmax_scale are
  *                            read; capacity and n_bins are filled in from the packing
  *   q_host                   host bf16 [T, Hq, D], tokens of prompt 0, then prompt 1, ...
@@ -278,8 +304,13 @@ int pp_decode_step(const pp_attn_params* params, const int32_t* lengths, int32_t
  * batches are one group, packed exactly as pp_pack packs the whole batch. The caches do not depend
  * on the grouping; O depends on it only through the position of tile boundaries (summation
  * order). Work already queued on `stream` is waited for first.
- * Errors: as the three calls it is made of, plus PP_ERR_DEVICE_TIMEOUT.
+ * pp_prefill_host_groups(n) fixes the number of groups for later calls of the calling thread
+ * (1 .. 16; 1 gives exactly the packing of pp_pack over the whole batch and with it O bit-identical
+ * to the device entry points; 0 restores the choice by batch size) and returns the previous setting;
+ * an n outside 0 .. 16 changes nothing.
+ * Errors: as pp_prefill_fused, plus PP_ERR_DEVICE_TIMEOUT.
  */
+int32_t pp_prefill_host_groups(int32_t n_groups);
 size_t pp_prefill_host_arena_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k);
 int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, int32_t k,
                     const void* q_host, const void* k_host, const void* v_host,

@@ -45,7 +45,7 @@ import math
 import numpy as np
 
 # --------------------------------------------------------------------------- #
-# Rotary positional encoding (reading A-7: rotate-half pairing)
+# Rotary positional encoding (rotate-half pairing)
 # --------------------------------------------------------------------------- #
 
 

@@ -14,6 +14,7 @@ _lib = None
 
 PP_FLAG_SKIP_ROPE = 1
 PP_FLAG_ROPE_ONLY = 2
+PP_FLAG_KEEP_ROPE_TABLE = 4
 
 
 class PrepackError(RuntimeError):
@@ -54,6 +55,7 @@ def load_library():
         "pp_last_cuda_error": (ctypes.c_char_p, []),
         "pp_pack": (ctypes.c_int, [i32p, ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p]),
         "pp_fill_position_ids": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, i32p, i32p]),
+        "pp_prefill_schedule_info": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, i32p]),
         "pp_prefill_workspace_bytes": (ctypes.c_size_t, [pp, ctypes.c_int32]),
         "pp_prefill_attention": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp,
                                                 ctypes.c_size_t, vp, vp]),
@@ -70,6 +72,7 @@ def load_library():
         "pp_decode_step": (ctypes.c_int, [pp, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp, i64p, i32p, vp, vp,
                                           ctypes.c_size_t, vp]),
         "pp_prefill_host_arena_bytes": (ctypes.c_size_t, [pp, i32p, ctypes.c_int32]),
+        "pp_prefill_host_groups": (ctypes.c_int32, [ctypes.c_int32]),
         "pp_prefill_host": (ctypes.c_int, [pp, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]),
     }
     for name, (res, args) in sig.items():
@@ -157,6 +160,20 @@ def pp_fill_position_ids(pack: Packing):
     return pos.reshape(pack.n_bins, pack.capacity), seg.reshape(pack.n_bins, pack.capacity)
 
 
+SCHEDULE_INFO_FIELDS = ("mode", "pairing", "entries", "steps", "key_tile_rows", "unpaired_entries",
+                        "late_joining_entries", "heads_folded")
+
+
+def pp_prefill_schedule_info(params: AttnParams, pack: Packing) -> dict:
+    """The tile work list pp_prefill_attention / pp_prefill_fused would build for this packing, as a
+    dict keyed by SCHEDULE_INFO_FIELDS (see include/pp.h)."""
+    info = np.zeros(8, np.int32)
+    st = load_library().pp_prefill_schedule_info(ctypes.byref(params), _p32(pack.bin_seg_ptr),
+                                                 _p32(pack.seg_start), _p32(pack.seg_len), pack.k, _p32(info))
+    _check(st, "pp_prefill_schedule_info")
+    return dict(zip(SCHEDULE_INFO_FIELDS, (int(x) for x in info)))
+
+
 def pp_prefill_workspace_bytes(params: AttnParams, k: int) -> int:
     return int(load_library().pp_prefill_workspace_bytes(ctypes.byref(params), k))
 
@@ -242,6 +259,12 @@ def pp_unpack_kv_static(params: AttnParams, bin_of, off_of, lengths, k_rot, v, k
 def pp_prefill_host_arena_bytes(params: AttnParams, lengths) -> int:
     l = _i32(lengths)
     return int(load_library().pp_prefill_host_arena_bytes(ctypes.byref(params), _p32(l), int(l.shape[0])))
+
+
+def pp_prefill_host_groups(n_groups: int) -> int:
+    """Fix the number of pipelined groups of pp_prefill_host for this thread (0 = by batch size);
+    returns the previous setting."""
+    return int(load_library().pp_prefill_host_groups(n_groups))
 
 
 def pp_prefill_host(params: AttnParams, lengths, q_host, k_host, v_host, o_host, k_cache_host, v_cache_host,

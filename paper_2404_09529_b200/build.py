@@ -11,7 +11,7 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libprepack_b200.so")
 SOURCES = ["pp_host.cpp", "pp_api.cu", "pp_rope.cu", "pp_attention.cu", "pp_unpack.cu", "pp_unpack_static.cu",
            "pp_tensorize.cu", "pp_decode.cu"]
-HEADERS = ["pp_internal.h", os.path.join("..", "..", "include", "pp.h")]
+HEADERS = ["pp_internal.h", "pp_device_once.h", os.path.join("..", "..", "include", "pp.h")]
 
 
 def _nvcc() -> str:

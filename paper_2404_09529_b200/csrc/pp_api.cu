@@ -4,7 +4,6 @@
 
 #include <algorithm>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -25,11 +24,12 @@ namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Internal flag bits (not part of the public header), used by pp_prefill_host to put the small table
-// uploads in front of its large data uploads: a table upload that is queued behind another
-// stream's bulk copy would hold its kernels back for milliseconds.
-constexpr int kFlagUploadOnly = 0x100;     // build and upload the tables, launch nothing
-constexpr int kFlagTablesReady = 0x200;    // the tables are in the workspace already: do not upload
+// What an entry point does with its tables. pp_prefill_host splits a call in two so that the small
+// table uploads go in front of its large data uploads: a table upload that is queued behind another
+// stream's bulk copy would hold its kernels back for milliseconds. Never reachable through
+// pp_attn_params.flags: the public entry points reject every bit they do not document.
+enum class TableStep { kUploadAndLaunch, kUploadOnly, kLaunchOnly };
+constexpr int kPublicFlags = PP_FLAG_SKIP_ROPE | PP_FLAG_ROPE_ONLY | PP_FLAG_KEEP_ROPE_TABLE;
 
 int check_params(const pp_attn_params* p) {
   if (!p) return PP_ERR_INVALID_ARG;
@@ -38,6 +38,7 @@ int check_params(const pp_attn_params* p) {
   if (p->n_q_heads % p->n_kv_heads != 0) return PP_ERR_UNSUPPORTED;
   if (p->n_kv_heads > 65535) return PP_ERR_UNSUPPORTED;
   if (!(p->rope_base > 0.f) || p->softmax_scale < 0.f) return PP_ERR_INVALID_ARG;
+  if (p->flags & ~kPublicFlags) return PP_ERR_INVALID_ARG;
   return PP_OK;
 }
 
@@ -94,12 +95,9 @@ extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t*
                                 static_cast<int32_t*>(host_workspace), workspace_bytes / sizeof(int32_t), &L);
   if (st != PP_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (!(flags & pp::kFlagTablesReady)) {
-    cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * (size_t)L.total_ints,
-                                    cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
-  }
-  if (flags & pp::kFlagUploadOnly) return PP_OK;
+  cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * (size_t)L.total_ints,
+                                  cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
   int32_t* d_table = static_cast<int32_t*>(workspace);
   if (do_rope) {
     st = pp::launch_rope(*params, d_table, L, q, q, k_, stream);
@@ -144,23 +142,53 @@ extern "C" size_t pp_prefill_fused_workspace_bytes(const pp_attn_params* params,
   return pp::fused_layout(*params, k).total_bytes;
 }
 
-extern "C" int pp_prefill_fused(const pp_attn_params* params, const int32_t* bin_seg_ptr,
-                                const int32_t* seg_start, const int32_t* seg_len, const int32_t* seg_prompt,
-                                int32_t k, const int32_t* lengths, const void* q, void* k_,
-                                const void* v, void* o, void* k_cache, void* v_cache, const int64_t* cache_off, const int32_t* cache_cap,
-                                void* workspace, void* host_workspace, size_t workspace_bytes,
-                                int32_t* device_status, void* stream) {
-  int st = pp::check_params(params);
+namespace pp {
+namespace {
+// The kernels of the fused path on tables that are (or will be, in stream order) in `workspace`.
+int launch_fused_kernels(const pp_attn_params& p, const TableLayout& L, const FusedLayout& f, const void* q,
+                         void* k_, const void* v, void* o, void* k_cache, void* v_cache, void* workspace,
+                         int32_t* device_status, void* stream) {
+  int st;
+  int32_t* d_table = static_cast<int32_t*>(workspace);
+  void* rope_table = static_cast<char*>(workspace) + f.off_rope_bytes;
+  if (!(p.flags & PP_FLAG_KEEP_ROPE_TABLE)) {
+    if ((st = launch_rope_table(p, rope_table, stream)) != PP_OK) return st;
+  }
+  if (!(p.flags & PP_FLAG_SKIP_ROPE)) {       // flag: k_ is rotated and the caches are filled already
+    st = launch_rope_unpack(p, d_table, L, (int32_t)f.off_true_len, (int32_t)f.off_cap,
+                            (int32_t)f.off_cache_off, rope_table, k_, v, k_cache, v_cache, stream);
+    if (st != PP_OK) return st;
+  }
+  if (p.flags & PP_FLAG_ROPE_ONLY) return PP_OK;
+  // the attention kernel rotates every Q tile in shared memory, so Q is read from HBM once
+  return launch_attention(p, d_table, L, q, k_, v, o, rope_table, device_status, stream);
+}
+
+// pp_prefill_fused, optionally cut in two: kUploadOnly validates, builds and uploads the tables,
+// launches nothing and hands the table layout back through `layout`; kLaunchOnly takes that layout,
+// touches neither the host staging buffer (its upload may still be in flight) nor the arguments
+// already checked, and launches the kernels on the tables in `workspace`.
+int prefill_fused_impl(const pp_attn_params* params, const int32_t* bin_seg_ptr, const int32_t* seg_start,
+                       const int32_t* seg_len, const int32_t* seg_prompt, int32_t k, const int32_t* lengths,
+                       const void* q, void* k_, const void* v, void* o, void* k_cache, void* v_cache,
+                       const int64_t* cache_off, const int32_t* cache_cap, void* workspace,
+                       void* host_workspace, size_t workspace_bytes, int32_t* device_status, void* stream,
+                       TableStep step, TableLayout* layout) {
+  int st = check_params(params);
   if (st != PP_OK) return st;
+  if (step == TableStep::kLaunchOnly) {
+    const FusedLayout f = fused_layout(*params, k);
+    return launch_fused_kernels(*params, *layout, f, q, k_, v, o, k_cache, v_cache, workspace, device_status, stream);
+  }
   if (!q || !k_ || !v || !o || !k_cache || !v_cache || !cache_off || !cache_cap || !seg_prompt || !lengths ||
       !workspace || !host_workspace)
     return PP_ERR_INVALID_ARG;
-  st = pp::validate_packing(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k);
+  st = validate_packing(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k);
   if (st != PP_OK) return st;
-  if (!pp::aligned16(q) || !pp::aligned16(k_) || !pp::aligned16(v) || !pp::aligned16(o) ||
-      !pp::aligned16(k_cache) || !pp::aligned16(v_cache) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+  if (!aligned16(q) || !aligned16(k_) || !aligned16(v) || !aligned16(o) ||
+      !aligned16(k_cache) || !aligned16(v_cache) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return PP_ERR_ALIGNMENT;
-  const pp::FusedLayout f = pp::fused_layout(*params, k);
+  const FusedLayout f = fused_layout(*params, k);
   if (workspace_bytes < f.total_bytes) return PP_ERR_BUFFER_TOO_SMALL;
   int32_t* h = static_cast<int32_t*>(host_workspace);
   int64_t* h_coff = reinterpret_cast<int64_t*>(h + f.off_cache_off);
@@ -174,26 +202,31 @@ extern "C" int pp_prefill_fused(const pp_attn_params* params, const int32_t* bin
     h[f.off_cap + s] = cache_cap[i];
     h_coff[s] = cache_off[i];
   }
-  if ((st = pp::check_device()) != PP_OK) return st;
-  pp::TableLayout L;
-  st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
-                                params->n_q_heads / params->n_kv_heads, h, f.table_ints, &L);
+  if ((st = check_device()) != PP_OK) return st;
+  TableLayout L;
+  st = build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
+                            params->n_q_heads / params->n_kv_heads, h, f.table_ints, &L);
   if (st != PP_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, sizeof(int32_t) * f.upload_ints,
                                   cudaMemcpyHostToDevice, s);
-  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "table upload");
-  int32_t* d_table = static_cast<int32_t*>(workspace);
-  void* rope_table = static_cast<char*>(workspace) + f.off_rope_bytes;
-  if ((st = pp::launch_rope_table(*params, rope_table, stream)) != PP_OK) return st;
-  if (!(params->flags & PP_FLAG_SKIP_ROPE)) {       // flag: k_ is rotated and the caches are filled already
-    st = pp::launch_rope_unpack(*params, d_table, L, (int32_t)f.off_true_len, (int32_t)f.off_cap,
-                                (int32_t)f.off_cache_off, rope_table, k_, v, k_cache, v_cache, stream);
-    if (st != PP_OK) return st;
-  }
-  if (params->flags & PP_FLAG_ROPE_ONLY) return PP_OK;
-  // the attention kernel rotates every Q tile in shared memory, so Q is read from HBM once
-  return pp::launch_attention(*params, d_table, L, q, k_, v, o, rope_table, device_status, stream);
+  if (e != cudaSuccess) return note_cuda_error((int)e, "table upload");
+  if (layout) *layout = L;
+  if (step == TableStep::kUploadOnly) return PP_OK;
+  return launch_fused_kernels(*params, L, f, q, k_, v, o, k_cache, v_cache, workspace, device_status, stream);
+}
+}  // namespace
+}  // namespace pp
+
+extern "C" int pp_prefill_fused(const pp_attn_params* params, const int32_t* bin_seg_ptr,
+                                const int32_t* seg_start, const int32_t* seg_len, const int32_t* seg_prompt,
+                                int32_t k, const int32_t* lengths, const void* q, void* k_,
+                                const void* v, void* o, void* k_cache, void* v_cache, const int64_t* cache_off, const int32_t* cache_cap,
+                                void* workspace, void* host_workspace, size_t workspace_bytes,
+                                int32_t* device_status, void* stream) {
+  return pp::prefill_fused_impl(params, bin_seg_ptr, seg_start, seg_len, seg_prompt, k, lengths, q, k_, v, o,
+                                k_cache, v_cache, cache_off, cache_cap, workspace, host_workspace, workspace_bytes,
+                                device_status, stream, pp::TableStep::kUploadAndLaunch, nullptr);
 }
 
 extern "C" int pp_selftest_bounded_wait(int32_t* device_status, uint32_t limit_ms, void* stream) {
@@ -250,12 +283,9 @@ extern "C" int pp_unpack_kv(const pp_attn_params* params, const int32_t* bin_of,
     h_coff[i] = cache_off[i];
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (!(params->flags & pp::kFlagTablesReady)) {
-    cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, pp::unpack_table_bytes(k),
-                                    cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return pp::note_cuda_error((int)e, "unpack table upload");
-  }
-  if (params->flags & pp::kFlagUploadOnly) return PP_OK;
+  cudaError_t e = cudaMemcpyAsync(workspace, host_workspace, pp::unpack_table_bytes(k),
+                                  cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return pp::note_cuda_error((int)e, "unpack table upload");
   return pp::launch_unpack(*params, static_cast<const int32_t*>(workspace), k, total, k_rot, v, k_cache,
                            v_cache, stream);
 }
@@ -268,7 +298,9 @@ namespace {
 
 size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
 
-constexpr int kHostGroups = 8;     // groups of prompts pp_prefill_host pipelines over its own streams
+constexpr int kHostGroupsMax = 16;     // groups of prompts pp_prefill_host can pipeline over its own streams
+constexpr int kHostGroupsDefault = 8;
+thread_local int g_host_groups = 0;    // pp_prefill_host_groups(); 0 = choose by batch size
 
 // How pp_prefill_host cuts a batch: contiguous ranges of prompts (original order) with about equal
 // token counts, each packed on its own with the batch-wide capacity, so that every tensor of a
@@ -285,7 +317,7 @@ struct HostPlan {
   std::vector<HostGroup> groups;
   // arena offsets (bytes)
   size_t q = 0, k = 0, v = 0, o = 0, q_tok = 0, k_tok = 0, v_tok = 0, o_tok = 0, kc = 0, vc = 0;
-  size_t ws_attn = 0, ws_attn_stride = 0, ws_unpack = 0, ws_unpack_stride = 0, map = 0, map_stride = 0;
+  size_t ws = 0, ws_stride = 0, map = 0, map_stride = 0;
   size_t status = 0, total = 0;
 };
 
@@ -301,11 +333,9 @@ int plan_host(const pp_attn_params& p, const int32_t* lengths, int32_t k, HostPl
   const size_t q_row = (size_t)p.n_q_heads * p.head_dim * 2, kv_row = (size_t)p.n_kv_heads * p.head_dim * 2;
   // pipelining pays once the transfers are tens of megabytes; small batches stay in one group
   const size_t batch_bytes = (size_t)h.total_tokens * (q_row + 2 * kv_row);
-  int n_groups = batch_bytes >= (size_t(32) << 20) ? std::min<int32_t>(kHostGroups, k) : 1;
-  if (const char* ev = std::getenv("PP_HOST_GROUPS")) {            // debug override
-    const int want = std::atoi(ev);
-    if (want >= 1) n_groups = std::min<int>(std::min<int>(want, kHostGroups), k);
-  }
+  int n_groups = batch_bytes >= (size_t(32) << 20) ? kHostGroupsDefault : 1;
+  if (g_host_groups > 0) n_groups = g_host_groups;
+  n_groups = std::min<int>(n_groups, k);
   h.groups.resize(n_groups);
   int32_t i = 0;
   int64_t t = 0;
@@ -342,12 +372,13 @@ int plan_host(const pp_attn_params& p, const int32_t* lengths, int32_t k, HostPl
   h.o_tok = off; off += up256(T * q_row);
   h.kc = off; off += up256(T * kv_row);
   h.vc = off; off += up256(T * kv_row);
-  // per-group tables, each sized for the whole batch (they are small)
-  h.ws_attn_stride = up256(sizeof(int32_t) * prefill_table_ints(h.n_bins, m, k));
-  h.ws_attn = off; off += n_groups * h.ws_attn_stride;
-  h.ws_unpack_stride = up256(unpack_table_bytes(k));
-  h.ws_unpack = off; off += n_groups * h.ws_unpack_stride;
-  h.map_stride = up256(sizeof(int64_t) * (2 * (size_t)k + 1));
+  // per-group workspace of the fused call, each sized for the whole batch (they are small)
+  pp_attn_params whole = p;
+  whole.capacity = m;
+  whole.n_bins = h.n_bins;
+  h.ws_stride = up256(fused_layout(whole, k).total_bytes);
+  h.ws = off; off += n_groups * h.ws_stride;
+  h.map_stride = up256(sizeof(int64_t) * (2 * (size_t)k + 1 + (size_t)h.n_bins));
   h.map = off; off += n_groups * h.map_stride;
   h.status = off; off += 256;
   h.total = off;
@@ -356,11 +387,11 @@ int plan_host(const pp_attn_params& p, const int32_t* lengths, int32_t k, HostPl
 
 // Streams and events pp_prefill_host pipelines over, created on first use per device.
 struct HostPipe {
-  cudaStream_t stream[kHostGroups] = {};
-  cudaEvent_t done[kHostGroups] = {};
+  cudaStream_t stream[kHostGroupsMax] = {};
+  cudaEvent_t done[kHostGroupsMax] = {};
   cudaEvent_t start = nullptr;
-  void* staging[kHostGroups] = {};        // pinned host staging for each group's tables
-  size_t staging_bytes[kHostGroups] = {};
+  void* staging[kHostGroupsMax] = {};        // pinned host staging for each group's tables
+  size_t staging_bytes[kHostGroupsMax] = {};
   int device = -1;
 };
 // Pinned staging of at least `bytes` for group g (kept and grown across calls; every call ends with a
@@ -387,14 +418,14 @@ int host_pipe(HostPipe** out) {
     // first use on this device (or a call that failed half-way): drop whatever an earlier device or
     // attempt left behind. Handles are destroyed with the device they were made on current.
     if (pipe.device >= 0 && cudaSetDevice(pipe.device) != cudaSuccess) (void)cudaGetLastError();
-    for (int g = 0; g < kHostGroups; ++g) {
+    for (int g = 0; g < kHostGroupsMax; ++g) {
       if (pipe.stream[g]) { cudaStreamDestroy(pipe.stream[g]); pipe.stream[g] = nullptr; }
       if (pipe.done[g]) { cudaEventDestroy(pipe.done[g]); pipe.done[g] = nullptr; }
     }
     if (pipe.start) { cudaEventDestroy(pipe.start); pipe.start = nullptr; }
     if (pipe.device >= 0 && (e = cudaSetDevice(dev)) != cudaSuccess) return note_cuda_error((int)e, "cudaSetDevice");
     pipe.device = -1;
-    for (int g = 0; g < kHostGroups; ++g) {
+    for (int g = 0; g < kHostGroupsMax; ++g) {
       if ((e = cudaStreamCreateWithFlags(&pipe.stream[g], cudaStreamNonBlocking)) != cudaSuccess)
         return note_cuda_error((int)e, "cudaStreamCreate");
       if ((e = cudaEventCreateWithFlags(&pipe.done[g], cudaEventDisableTiming)) != cudaSuccess)
@@ -410,6 +441,12 @@ int host_pipe(HostPipe** out) {
 
 }  // namespace
 }  // namespace pp
+
+extern "C" int32_t pp_prefill_host_groups(int32_t n_groups) {
+  const int32_t before = pp::g_host_groups;
+  if (n_groups >= 0 && n_groups <= pp::kHostGroupsMax) pp::g_host_groups = n_groups;
+  return before;
+}
 
 extern "C" size_t pp_prefill_host_arena_bytes(const pp_attn_params* params, const int32_t* lengths, int32_t k) {
   if (!params || !lengths || k < 1) return 0;
@@ -449,44 +486,44 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
     const size_t q_row = (size_t)params->n_q_heads * params->head_dim * 2;
     const size_t kv_row = (size_t)params->n_kv_heads * params->head_dim * 2;
     cudaError_t e;
-#define PP_TRY(call, what) do { e = (call); if (e != cudaSuccess) return pp::note_cuda_error((int)e, what); } while (0)
-    // Every group runs on its own stream: one upload per tensor, TENSORIZE on the device, the three
-    // kernels of the path, O gathered back to token order, one download per tensor. The uploads of
-    // one group overlap the kernels of another and the downloads of a third (PCIe is full duplex).
+    // Every group runs on its own stream: one upload per tensor, TENSORIZE on the device, the two
+    // kernels of the fused path (which write the caches in token order), O gathered back to token
+    // order, one download per tensor. The uploads of one group overlap the kernels of another and
+    // the downloads of a third (PCIe is full duplex).
     pp::HostPipe* pipe = nullptr;
     if ((st = pp::host_pipe(&pipe)) != PP_OK) return st;
     // On an error in the middle of the pipeline, work already queued on the internal streams still
     // reads and writes the caller's buffers: wait for it before handing the error back.
     auto bail = [&](int code) {
-      for (int g = 0; g < pp::kHostGroups; ++g) (void)cudaStreamSynchronize(pipe->stream[g]);
+      for (int g = 0; g < pp::kHostGroupsMax; ++g) (void)cudaStreamSynchronize(pipe->stream[g]);
       (void)cudaStreamSynchronize(s);
       return code;
     };
-#undef PP_TRY
 #define PP_TRY(call, what) do { e = (call); if (e != cudaSuccess) return bail(pp::note_cuda_error((int)e, what)); } while (0)
     const int n_groups = (int)h.groups.size();
     PP_TRY(cudaMemsetAsync(base + h.status, 0, 4, s), "memset status");
     PP_TRY(cudaEventRecord(pipe->start, s), "event record");
     std::vector<int64_t> g_cache_off;
-    const bool trace = std::getenv("PP_HOST_TRACE") != nullptr;      // debug: print each group's timeline
-    std::vector<cudaEvent_t> tev;
-    auto mark = [&](cudaStream_t st_) { if (trace) { cudaEvent_t ev; cudaEventCreate(&ev); cudaEventRecord(ev, st_); tev.push_back(ev); } };
-    mark(s);
+    int32_t* d_status = reinterpret_cast<int32_t*>(base + h.status);
     for (int g = 0; g < n_groups; ++g) {
       const pp::HostGroup& G = h.groups[g];
       const int32_t kg = G.i1 - G.i0;
       const size_t tok0 = (size_t)G.t0, ntok = (size_t)(G.t1 - G.t0);
-      const size_t rows0 = (size_t)G.bin0 * cap, nrows = (size_t)G.n_bins * cap;
+      const size_t rows0 = (size_t)G.bin0 * cap;
       cudaStream_t sg = pipe->stream[g];
       PP_TRY(cudaStreamWaitEvent(sg, pipe->start, 0), "stream wait");
-      // The small uploads first (token -> packed row map and the two tables of the group, from pinned
-      // staging): queued behind another group's bulk copies they would hold this group's kernels back.
-      const size_t map_bytes = (sizeof(int64_t) * (2 * (size_t)kg + 1) + 255) & ~size_t(255);
-      const size_t attn_tab = (sizeof(int32_t) * pp::prefill_table_ints(G.n_bins, cap, kg) + 255) & ~size_t(255);
-      const size_t unpack_tab = (pp::unpack_table_bytes(kg) + 255) & ~size_t(255);
+      // The small uploads first (token -> packed row map, rows used per bin, and the group's tables,
+      // from pinned staging): queued behind another group's bulk copies they would hold this group's
+      // kernels back for milliseconds.
+      pp_attn_params gp = *params;
+      gp.n_bins = G.n_bins;
+      const size_t map_ints64 = 2 * (size_t)kg + 1 + (size_t)G.n_bins;
+      const size_t map_bytes = pp::up256(sizeof(int64_t) * map_ints64);
+      const size_t tab_bytes = pp::up256(pp::fused_layout(gp, kg).total_bytes);
       void* stage = nullptr;
-      if ((st = pp::host_staging(pipe, g, map_bytes + attn_tab + unpack_tab, &stage)) != PP_OK) return bail(st);
+      if ((st = pp::host_staging(pipe, g, map_bytes + tab_bytes, &stage)) != PP_OK) return bail(st);
       int64_t* map = static_cast<int64_t*>(stage);
+      int64_t* used = map + 2 * (size_t)kg + 1;
       g_cache_off.resize(kg);
       int64_t t = 0;
       for (int32_t j = 0; j < kg; ++j) {
@@ -496,73 +533,53 @@ extern "C" int pp_prefill_host(pp_attn_params* params, const int32_t* lengths, i
         t += lengths[G.i0 + j];
       }
       map[kg] = t;
+      for (int32_t b = 0; b < G.n_bins; ++b) {
+        const int32_t last = G.bin_seg_ptr[b + 1] - 1;
+        used[b] = (int64_t)G.seg_start[last] + G.seg_len[last];
+      }
       int64_t* d_map = reinterpret_cast<int64_t*>(base + h.map + g * h.map_stride);
-      PP_TRY(cudaMemcpyAsync(d_map, map, sizeof(int64_t) * (2 * (size_t)kg + 1), cudaMemcpyHostToDevice, sg), "H2D map");
+      PP_TRY(cudaMemcpyAsync(d_map, map, sizeof(int64_t) * map_ints64, cudaMemcpyHostToDevice, sg), "H2D map");
       char* gq = base + h.q + rows0 * q_row;
       char* gk = base + h.k + rows0 * kv_row;
       char* gv = base + h.v + rows0 * kv_row;
       char* go = base + h.o + rows0 * q_row;
-      pp_attn_params gp = *params;
-      gp.n_bins = G.n_bins;
-      gp.flags = pp::kFlagUploadOnly;
-      st = pp_prefill_attention(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), kg, gq, gk, gv, go,
-                                base + h.ws_attn + g * h.ws_attn_stride, static_cast<char*>(stage) + map_bytes, attn_tab,
-                                reinterpret_cast<int32_t*>(base + h.status), sg);
+      char* gws = base + h.ws + g * h.ws_stride;
+      void* gstage = static_cast<char*>(stage) + map_bytes;
+      pp::TableLayout g_layout;
+      st = pp::prefill_fused_impl(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), G.seg_prompt.data(),
+                                  kg, lengths + G.i0, gq, gk, gv, go, base + h.kc, base + h.vc, g_cache_off.data(),
+                                  lengths + G.i0, gws, gstage, tab_bytes, d_status, sg, pp::TableStep::kUploadOnly, &g_layout);
       if (st != PP_OK) return bail(st);
-      st = pp_unpack_kv(&gp, G.bin_of.data(), G.off_of.data(), lengths + G.i0, kg, gk, gv, base + h.kc, base + h.vc,
-                        g_cache_off.data(), lengths + G.i0, base + h.ws_unpack + g * h.ws_unpack_stride,
-                        static_cast<char*>(stage) + map_bytes + attn_tab, unpack_tab, sg);
-      if (st != PP_OK) return bail(st);
-      gp.flags = pp::kFlagTablesReady;
       PP_TRY(cudaMemcpyAsync(base + h.q_tok + tok0 * q_row, (const char*)q_host + tok0 * q_row, ntok * q_row,
                              cudaMemcpyHostToDevice, sg), "H2D q");
       PP_TRY(cudaMemcpyAsync(base + h.k_tok + tok0 * kv_row, (const char*)k_host + tok0 * kv_row, ntok * kv_row,
                              cudaMemcpyHostToDevice, sg), "H2D k");
       PP_TRY(cudaMemcpyAsync(base + h.v_tok + tok0 * kv_row, (const char*)v_host + tok0 * kv_row, ntok * kv_row,
                              cudaMemcpyHostToDevice, sg), "H2D v");
-      mark(sg);
-      // padding rows of the packed buffers must be finite
-      PP_TRY(cudaMemsetAsync(base + h.q + rows0 * q_row, 0, nrows * q_row, sg), "memset packed q");
-      PP_TRY(cudaMemsetAsync(base + h.k + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed k");
-      PP_TRY(cudaMemsetAsync(base + h.v + rows0 * kv_row, 0, nrows * kv_row, sg), "memset packed v");
-      mark(sg);   // memsets
+      // TENSORIZE: padding rows of the packed tensors zeroed (they must be finite), real rows scattered
+      if ((st = pp::launch_zero_pad_rows(gq, gk, gv, (int32_t)q_row, (int32_t)kv_row, d_map + 2 * (size_t)kg + 1,
+                                         G.n_bins, cap, sg)) != PP_OK) return bail(st);
       if ((st = pp::launch_tensorize(true, gq, base + h.q_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return bail(st);
       if ((st = pp::launch_tensorize(true, gk, base + h.k_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return bail(st);
       if ((st = pp::launch_tensorize(true, gv, base + h.v_tok + tok0 * kv_row, d_map, kg, (int64_t)ntok, (int32_t)kv_row, sg)) != PP_OK) return bail(st);
-      mark(sg);   // scatter
-      st = pp_prefill_attention(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), kg, gq, gk, gv, go,
-                                base + h.ws_attn + g * h.ws_attn_stride, static_cast<char*>(stage) + map_bytes, attn_tab,
-                                reinterpret_cast<int32_t*>(base + h.status), sg);
+      st = pp::prefill_fused_impl(&gp, G.bin_seg_ptr.data(), G.seg_start.data(), G.seg_len.data(), G.seg_prompt.data(),
+                                  kg, lengths + G.i0, gq, gk, gv, go, base + h.kc, base + h.vc, g_cache_off.data(),
+                                  lengths + G.i0, gws, gstage, tab_bytes, d_status, sg, pp::TableStep::kLaunchOnly, &g_layout);
       if (st != PP_OK) return bail(st);
-      mark(sg);   // attention
-      st = pp_unpack_kv(&gp, G.bin_of.data(), G.off_of.data(), lengths + G.i0, kg, gk, gv, base + h.kc, base + h.vc,
-                        g_cache_off.data(), lengths + G.i0, base + h.ws_unpack + g * h.ws_unpack_stride,
-                        static_cast<char*>(stage) + map_bytes + attn_tab, unpack_tab, sg);
-      if (st != PP_OK) return bail(st);
+      // the caches are final once the first kernel of the fused path has run; O follows the attention
       if ((st = pp::launch_tensorize(false, go, base + h.o_tok + tok0 * q_row, d_map, kg, (int64_t)ntok, (int32_t)q_row, sg)) != PP_OK) return bail(st);
-      mark(sg);
-      PP_TRY(cudaMemcpyAsync((char*)o_host + tok0 * q_row, base + h.o_tok + tok0 * q_row, ntok * q_row,
-                             cudaMemcpyDeviceToHost, sg), "D2H o");
       PP_TRY(cudaMemcpyAsync((char*)k_cache_host + tok0 * kv_row, base + h.kc + tok0 * kv_row, ntok * kv_row,
                              cudaMemcpyDeviceToHost, sg), "D2H k cache");
       PP_TRY(cudaMemcpyAsync((char*)v_cache_host + tok0 * kv_row, base + h.vc + tok0 * kv_row, ntok * kv_row,
                              cudaMemcpyDeviceToHost, sg), "D2H v cache");
-      mark(sg);
+      PP_TRY(cudaMemcpyAsync((char*)o_host + tok0 * q_row, base + h.o_tok + tok0 * q_row, ntok * q_row,
+                             cudaMemcpyDeviceToHost, sg), "D2H o");
       PP_TRY(cudaEventRecord(pipe->done[g], sg), "event record");
       PP_TRY(cudaStreamWaitEvent(s, pipe->done[g], 0), "stream wait");
     }
     int32_t status = 0;
     PP_TRY(cudaMemcpyAsync(&status, base + h.status, 4, cudaMemcpyDeviceToHost, s), "D2H status");
     PP_TRY(cudaStreamSynchronize(s), "stream synchronize");
-    if (trace) {
-      for (size_t i = 1; i < tev.size(); ++i) {
-        float ms = 0.f;
-        cudaEventElapsedTime(&ms, tev[0], tev[i]);
-        std::fprintf(stderr, "%s%.2f", (i - 1) % 6 == 0 ? "\n[pp_prefill_host] group: h2d, memset, scatter, attention, unpack+gather, d2h done (ms): " : ", ", ms);
-      }
-      std::fprintf(stderr, "\n");
-      for (cudaEvent_t ev : tev) cudaEventDestroy(ev);
-    }
 #undef PP_TRY
     return status == 0 ? PP_OK : PP_ERR_DEVICE_TIMEOUT;
   } catch (const std::bad_alloc&) {

@@ -41,6 +41,7 @@
 #include <cstdlib>
 #include <type_traits>
 
+#include "pp_device_once.h"
 #include "pp_internal.h"
 
 namespace pp {
@@ -266,18 +267,6 @@ __host__ __device__ constexpr uint32_t instr_desc(uint32_t n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) |
          ((128u >> 4) << 24);
 }
-
-#ifdef PP_PROFILE
-// Debug-only cycle accounting (separate build with -DPP_PROFILE; not part of the product library).
-__device__ long long g_prof[160 * 32];
-#define PROF_DECL(n) long long prof_acc[n] = {}; long long prof_t = clock64()
-#define PROF_LAP(i) do { const long long now_ = clock64(); prof_acc[i] += now_ - prof_t; prof_t = now_; } while (0)
-#define PROF_STORE(base, n) do { if (blockIdx.x < 160) for (int i_ = 0; i_ < (n); ++i_) g_prof[blockIdx.x * 32 + (base) + i_] = prof_acc[i_]; } while (0)
-#else
-#define PROF_DECL(n)
-#define PROF_LAP(i)
-#define PROF_STORE(base, n)
-#endif
 
 struct AttnArgs {
   const int32_t* table;
@@ -533,12 +522,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t b_q_empty = bar_q_empty + 8 * t;
         uint32_t it_n = 0, kc = 0;       // items and key tiles consumed
         bool ok = true;
-        PROF_DECL(8);
         // S(kq) = Q_t K(kq)^T into buffer kq & 1
         auto issue_qk = [&](const uint32_t kq, const bool last_of_item) -> bool {
           const uint32_t b = kq & 1u;
           if (!mbar_wait(b_k_full + 8 * b, (kq >> 1) & 1u, wctx, kWaitKFull)) return false;
-          PROF_LAP(2);
           tc_fence_after();
           const uint32_t d = tm_s + 64u * b;
           const uint32_t kb = k_lo + b * (Cfg::kKVBytes >> 4);
@@ -551,7 +538,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           tc_commit(b_k_empty + 8 * b);
           tc_commit(b_s_full + 8 * b);
           if (last_of_item) tc_commit(b_q_empty);     // last read of Q_t in this item
-          PROF_LAP(3);
           return true;
         };
         // The slot's tiles form one stream across items: while the softmax threads work on tile k,
@@ -566,7 +552,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             mbar_arrive(b_item_empty);
           }
         }
-        PROF_LAP(0);
         if (ok && w >= 0) ok = mbar_wait(bar_q_ready, 0u, wctx, kWaitQFull) && issue_qk(kc, n == 1);
         while (ok && w >= 0) {
           const bool last_tile = (j + 1 == n);
@@ -577,26 +562,20 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (j == 0 && last_tile && !(ok = mbar_wait(b_o_empty, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
           if (last_tile) {
             const uint32_t item = it_n + 1u, ring = item % kRing;
-            PROF_LAP(4);
             if (!(ok = mbar_wait(b_item_full + 8 * ring, (item / kRing) & 1u, wctx, kWaitItemFull))) break;
             const volatile int* e = s_ring + (t * (int)kRing + (int)ring) * kRingInts;
             w_next = e[0]; n_next = e[3];
             mbar_arrive(b_item_empty + 8 * ring);
-            PROF_LAP(0);
             have = w_next >= 0;
             last_flag = n_next == 1;
             if (have && !(ok = mbar_wait(bar_q_ready, item & 1u, wctx, kWaitQFull))) break;
-            PROF_LAP(1);
           }
           if (have && !(ok = issue_qk(kc + 1, last_flag))) break;
           // the previous item's epilogue must have read O_t before it is overwritten
           if (j == 0 && !last_tile && !(ok = mbar_wait(b_o_empty, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty))) break;
-          PROF_LAP(4);
           const uint32_t b = kc & 1u, parity = (kc >> 1) & 1u;
           if (!(ok = mbar_wait(b_p_full + 8 * b, parity, wctx, kWaitP))) break;
-          PROF_LAP(5);
           if (!(ok = mbar_wait(b_v_full + 8 * b, parity, wctx, kWaitVFull))) break;
-          PROF_LAP(6);
           tc_fence_after();            // O_t (+)= P(k) V(k)
           const uint32_t a = tm_s + 64u * b;
           const uint32_t vb = v_lo + b * (Cfg::kKVBytes >> 4);
@@ -605,7 +584,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int kk = 1; kk < BN / 16; ++kk)
             mma_ts(tm_o, a + kk * 8, vb + (uint32_t)kk * ((16 * 128) >> 4), idesc_pv, 1u);
           tc_commit(b_v_empty + 8 * b);
-          PROF_LAP(7);
           ++kc;
           if (last_tile) {
             tc_commit(b_o_full);
@@ -615,7 +593,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ++j;
           }
         }
-        if (t == 0) PROF_STORE(0, 8);
       }
     } else {
     if (warp == 0 && lane == 0) {
@@ -692,13 +669,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       uint32_t it_n = 0, kc0 = 0, vc0 = 0, tc0 = 0, tc1 = 0;
       int n = 0, je0 = 0, jb1 = 0, je1 = 0;
       bool ok = true;
-      PROF_DECL(8);
       // S_t = Q_t K_j^T; the K stage is released after the last slot that reads it
       auto issue_qk = [&](const int t, const int j) -> bool {
         const uint32_t kc = kc0 + (uint32_t)j, s = kc % NK;
-        PROF_LAP(7);
         if (!mbar_wait(bar_k_full + 8 * s, (kc / NK) & 1u, wctx, kWaitKFull)) return false;
-        PROF_LAP(2);
         tc_fence_after();
         const uint32_t d = tmem_base + Cfg::kTmemS + 128u * t;
         const uint32_t a_lo = q_lo0 + (uint32_t)t * (Cfg::kQBytes >> 4);
@@ -711,22 +685,17 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         if (t == 1 || !(j >= jb1 && j < je1)) tc_commit(bar_k_empty + 8 * s);
         tc_commit(bar_s_full + 16 * t);
-        PROF_LAP(3);
         return true;
       };
       // O_t (+)= P_t V_j, then either the next S_t or the end-of-item signals of slot t
       auto slot_step = [&](const int t, const int j, const int jb, const int je, uint32_t& tcount) -> bool {
         if (j >= jb && j < je) {
           const bool first = (j == jb);
-          PROF_LAP(7);
           // the previous item's epilogue must have read O_t before it is overwritten
           if (first && !mbar_wait(bar_o_empty + 8 * t, (it_n & 1u) ^ 1u, wctx, kWaitOEmpty)) return false;
-          PROF_LAP(4);
           if (!mbar_wait(bar_p_full + 16 * t, tcount & 1u, wctx, kWaitP)) return false;
-          PROF_LAP(5);
           const uint32_t vc = vc0 + (uint32_t)j, s = vc % NV;
           if (!mbar_wait(bar_v_full + 8 * s, (vc / NV) & 1u, wctx, kWaitVFull)) return false;
-          PROF_LAP(6);
           tc_fence_after();
           const uint32_t a = tmem_base + Cfg::kTmemS + 128u * t;
           const uint32_t d = tmem_base + Cfg::kTmemO + (uint32_t)D * t;
@@ -747,19 +716,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       };
       while (ok) {
         const uint32_t ring = it_n % kRing;
-        PROF_LAP(7);
         if (!mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull)) break;
         const volatile int* e = s_ring + ring * kRingInts;
         const int w = e[0];
         n = e[3]; jb1 = e[6]; je0 = e[7]; je1 = e[8];
         mbar_arrive(bar_item_empty + 8 * ring);
         if (w < 0) break;
-        PROF_LAP(0);
         const uint32_t bar_q_ready = args.rope_table ? bar_q_rot : bar_q_full;
         ok = mbar_wait(bar_q_ready + 0, it_n & 1u, wctx, kWaitQFull) &&
              mbar_wait(bar_q_ready + 8, it_n & 1u, wctx, kWaitQFull);
         if (!ok) break;
-        PROF_LAP(1);
         if (je0 > 0) ok = issue_qk(0, 0);
         if (ok && jb1 == 0 && je1 > 0) ok = issue_qk(1, 0);
         for (int j = 0; ok && j < n; ++j) {
@@ -784,7 +750,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         vc0 += (uint32_t)n;
         ++it_n;
       }
-      PROF_STORE(0, 8);
     }
     }   // shared-stream roles
   } else {
@@ -822,12 +787,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (h == 0) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxIndep));
         uint32_t it_n = 0, tcount = 0;
-        PROF_DECL(12);
         while (true) {
           const uint32_t ring = ring0 + it_n % kRing;
-          PROF_LAP(8);
           ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull));
-          PROF_LAP(0);
           if (!ok) break;
           const volatile int* e = s_ring + ring * kRingInts;
           const int w = e[0], item_kv_row0 = e[2], n_tiles = e[3];
@@ -837,7 +799,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (w < 0) break;
           float m_run = -INFINITY;      // running maximum of the row, in scaled log2 units
           float l_run = 0.f;            // running sum of exp2(s * c - m_run)
-          PROF_LAP(8);
           for (int j = 0; j < n_tiles; ++j) {
             constexpr int EPT = BN;                              // scores per thread and tile
             constexpr int NCH = EPT / 32;                        // 32-column TMEM round trips
@@ -854,11 +815,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const bool cut_hi = (warp_flags & 4u) != 0, cut_lo = (warp_flags & 8u) != 0;
             const uint32_t sbuf = tcount & 1u;                   // tile k of the stream lives in S buffer k & 1
             const uint32_t tmem_sb = tmem_s + 64u * sbuf;
-            PROF_LAP(5);
             ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * (2 * t + sbuf), (tcount >> 1) & 1u, wctx, kWaitS));
             if (!ok) break;
             tc_fence_after();
-            PROF_LAP(1);
             uint32_t v[EPT];
 #pragma unroll
             for (int ch = 0; ch < NCH; ++ch) {
@@ -870,7 +829,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               }
             }
             tc_wait_ld();
-            PROF_LAP(2);
             // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
             // one of the two bounds (the causal diagonal, or the first tile of a prompt)
             if (cut_hi) {
@@ -898,7 +856,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               m1 = fmax3(m1, __uint_as_float(v[EPT - 2]), __uint_as_float(v[EPT - 1]));
               mx = fmaxf(fmax3(m0, m1, m2), m3);
             }
-            PROF_LAP(3);
             // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
             const float m_tile = mx * c_scale;
             float m_new = m_run;
@@ -922,7 +879,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tmem_st16(tmem_o + ch * 16, ov);
               }
             }
-            PROF_LAP(9);
             l_run *= alpha;
             m_run = m_new;
             const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
@@ -955,7 +911,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             float sum0, sum1, sum2, sum3;
             unpack_f2(sum_a, sum0, sum1);
             unpack_f2(sum_b, sum2, sum3);
-            PROF_LAP(4);
             l_run += (sum0 + sum2) + (sum1 + sum3);
             tc_wait_st();
             tc_fence_before();
@@ -969,13 +924,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // hand-over is double-buffered by item parity, barrier included.
           x_l[256 * (it_n & 1u)] = l_run;
           mbar_arrive(bar_l_ready + 16 * t + 8 * (it_n & 1u));
-          PROF_LAP(7);
           ++it_n;
         }
-#ifdef PP_PROFILE
-        prof_acc[10] = tcount;
-        if (row == 0) PROF_STORE(8 + 12 * t, 12);
-#endif
       } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsHelper));
         uint32_t it_n = 0;
@@ -1108,13 +1058,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int32_t* tb = args.table;
     uint32_t it_n = 0, tcount = 0;
     bool ok = true;
-    PROF_DECL(12);
     // Rotates this thread's part of row `row` of Q_t in shared memory by the angles of position
     // `pos` (<= 0: nothing to do), with the same fp32 arithmetic and rounding as the stand-alone
     // kernel, then reports the slot's Q as ready. Waits for the TMA load of Q first.
     auto rotate_q = [&](const int pos, const uint32_t parity) -> bool {
       if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * t, parity, wctx, kWaitQFull))) return false;
-      PROF_LAP(8);
       if (pos > 0) {
         constexpr int kUnits = D / 16;                 // 16-byte units per half of a row
         const uint32_t q_row = s_q + (uint32_t)t * Cfg::kQBytes + (uint32_t)row * 128;
@@ -1157,9 +1105,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // in independent mode slot t has its own ring, and an item describes one tile (its slot-0 fields)
       const uint32_t ring = it_n % kRing;
       const int f = t;                                 // which slot fields of the entry to read
-      PROF_LAP(8);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_item_full + 8 * ring, (it_n / kRing) & 1u, wctx, kWaitItemFull));
-      PROF_LAP(0);
       if (!ok) break;
       const volatile int* e = s_ring + ring * kRingInts;
       const int w = e[0];
@@ -1179,12 +1125,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           lo = seg_start_at(tb + args.off_seg_start, seg_first_t + 1, seg_end, i_row, lo, lane);
         if (i_row < bin_used) { key_lo = lo; key_hi = i_row; }
       }
-      PROF_LAP(8);
       // Fused path: Q arrives raw and is rotated in shared memory.
       if (args.rope_table) {
         ok = rotate_q(used ? key_hi - key_lo : -1, it_n & 1u);
         if (!ok) break;
-        PROF_LAP(11);
       }
       float m_run = -INFINITY;      // running maximum of the whole row, in scaled log2 units
       float l_run = 0.f;            // this thread's share of the running sum of exp2(s * c - m_run)
@@ -1206,11 +1150,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t sbuf = 0u;
         const uint32_t tparity = tcount & 1u;
         const uint32_t tmem_sb = tmem_s;
-        PROF_LAP(5);
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * (2 * t + sbuf), tparity, wctx, kWaitS));
         if (!ok) break;                                      // warp-uniform
         tc_fence_after();
-        PROF_LAP(1);
 
         // this thread's scores
         uint32_t v[EPT];
@@ -1224,7 +1166,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         tc_wait_ld();
-        PROF_LAP(2);
         // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
         // one of the two bounds (the causal diagonal, or the first tile of a prompt)
         if (cut_hi) {
@@ -1258,7 +1199,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         *x_mine = mx;
         if (!(ok = rendezvous(bar_pair, pair_ph, kWaitPair))) break;
         mx = fmaxf(mx, *x_other);
-        PROF_LAP(3);
         // lazy running-maximum update: keep the stale maximum while the new one is < 2^8 above it
         const float m_tile = mx * c_scale;
         float m_new = m_run;
@@ -1278,7 +1218,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tmem_st16(tmem_o + (D / 2) * h + ch * 16, ov);
           }
         }
-        PROF_LAP(9);
         l_run *= alpha;
         m_run = m_new;
         const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
@@ -1311,7 +1250,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         float sum0, sum1, sum2, sum3;
         unpack_f2(sum_a, sum0, sum1);
         unpack_f2(sum_b, sum2, sum3);
-        PROF_LAP(4);
         l_run += (sum0 + sum2) + (sum1 + sum3);
         tc_wait_st();
         tc_fence_before();
@@ -1321,10 +1259,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (!ok) break;
 
       // epilogue: O_t / l -> bf16 -> shared memory (128-byte swizzle) -> TMA store
-      PROF_LAP(5);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_o_full + 8 * t, it_n & 1u, wctx, kWaitOFull));
       if (!ok) break;
-      PROF_LAP(6);
       if (used) {
         // the half-1 threads hand their share of the row sum to the half-0 threads, which run the
         // epilogue; the second barrier keeps the exchange slot from being reused too early
@@ -1374,14 +1310,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         mbar_arrive(bar_o_empty + 8 * t);
       }
       if (!ok) break;
-      PROF_LAP(7);
       ++it_n;
     }
     if (h == 0 && lane == 0) tma_store_wait_read();    // staging must outlive the last store's read
-#ifdef PP_PROFILE
-    prof_acc[10] = tcount;
-    if (row == 0 && h == 0) PROF_STORE(8 + 12 * t, 12);
-#endif
     }   // shared-stream mode
   }
 
@@ -1484,12 +1415,15 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   if ((st = make_map(&mk, k, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
   if ((st = make_map(&mv, v, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
   if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, 32)) != PP_OK) return st;   // one warp's rows per store
-  static bool configured = false;   // per process, per template instance
-  if (!configured) {
+  // the shared-memory opt-in of a kernel is a per-device attribute
+  static DeviceOnce configured;     // per template instance
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return note_cuda_error(-1, "cudaGetDevice");
+  if (!configured.done(dev)) {
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<D, kIndep>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Cfg::kSmemBytes);
     if (e != cudaSuccess) return note_cuda_error((int)e, "cudaFuncSetAttribute(smem)");
-    configured = true;
+    configured.mark(dev);
   }
   const int sms = sm_count();
   if (sms <= 0) return note_cuda_error(-1, "multiprocessor count");
@@ -1529,12 +1463,6 @@ int launch_bounded_wait_selftest(int32_t* device_status, uint64_t limit_ns, void
   const cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "self-test kernel launch");
 }
-
-#ifdef PP_PROFILE
-extern "C" int pp_debug_read_profile(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_prof, sizeof(long long) * (size_t)n);
-}
-#endif
 
 int launch_attention(const pp_attn_params& p, int32_t* d_table, const TableLayout& L, const void* q,
                      const void* k, const void* v, void* o, const void* rope_table, int32_t* device_status,

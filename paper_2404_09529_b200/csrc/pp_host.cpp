@@ -175,7 +175,7 @@ namespace pp {
 
 size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k) {
   const int64_t q_tiles = (int64_t)n_bins * ((capacity + kTileM - 1) / kTileM);
-  // header + bin_seg_ptr + bin_used + seg_start + items (8 ints each), each block 4-int aligned
+  // header + bin_seg_ptr + bin_used + seg_start + items (kItemInts ints each), each block 4-int aligned
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
   return (size_t)(kHeaderInts + up4(n_bins + 1) + up4(n_bins) + up4(k) + kItemInts * q_tiles);
 }
@@ -299,8 +299,45 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   out[kHeaderCounter] = 0;   // work counter the CTAs draw from; reset by every upload
   L.total_ints = (int32_t)(L.items + kItemInts * (int64_t)items.size());
   L.independent_slots = independent;
+  L.pair_rows = pair_rows;
   if (layout) *layout = L;
   return PP_OK;
 }
 
 }  // namespace pp
+
+extern "C" int pp_prefill_schedule_info(const pp_attn_params* params, const int32_t* bin_seg_ptr,
+                                        const int32_t* seg_start, const int32_t* seg_len, int32_t k,
+                                        int32_t* info) {
+  if (!params || !info) return PP_ERR_INVALID_ARG;
+  if (params->n_q_heads < 1 || params->n_kv_heads < 1) return PP_ERR_INVALID_ARG;
+  if (params->n_q_heads % params->n_kv_heads != 0) return PP_ERR_UNSUPPORTED;
+  int st = pp::validate_packing(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k);
+  if (st != PP_OK) return st;
+  try {
+    std::vector<int32_t> table(pp::prefill_table_ints(params->n_bins, params->capacity, k));
+    pp::TableLayout L;
+    st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
+                                  params->n_q_heads / params->n_kv_heads, table.data(), table.size(), &L);
+    if (st != PP_OK) return st;
+    const pp::WorkItem* items = reinterpret_cast<const pp::WorkItem*>(table.data() + L.items);
+    int64_t steps = 0;
+    int32_t unpaired = 0, late = 0;
+    for (int32_t i = 0; i < L.n_items; ++i) {
+      steps += items[i].cost;
+      if (items[i].q_row0[1] < 0) ++unpaired;
+      else if (items[i].jb1 > 0) ++late;
+    }
+    info[0] = L.independent_slots ? 1 : 0;
+    info[1] = L.independent_slots ? 2 : (L.pair_rows ? 1 : 0);
+    info[2] = L.n_items;
+    info[3] = (int32_t)std::min<int64_t>(steps, INT32_MAX);
+    info[4] = L.independent_slots ? pp::kTileNShort : pp::kTileN;
+    info[5] = unpaired;
+    info[6] = late;
+    info[7] = 1;
+  } catch (const std::bad_alloc&) {
+    return PP_ERR_NO_MEMORY;
+  }
+  return PP_OK;
+}

@@ -43,6 +43,7 @@ struct TableLayout {
   int32_t n_items = 0;
   int32_t total_ints = 0;
   bool independent_slots = false;   // items are single tiles, drawn by each slot on its own
+  bool pair_rows = false;           // shared-stream mode: the two slots are consecutive row tiles of one head
 };
 
 int validate_packing(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
@@ -79,6 +80,10 @@ int launch_unpack(const pp_attn_params& p, const int32_t* d_table, int32_t k, in
 // d_map: device int64 tok_prefix[n_prompts + 1] followed by first_row[n_prompts].
 int launch_tensorize(bool to_packed, void* packed, void* tokens, const int64_t* d_map, int32_t n_prompts,
                      int64_t total_tokens, int32_t row_bytes, void* stream);
+
+// Zeroes rows [bin_used[b], capacity) of every bin of the packed q / k / v (null pointers are skipped).
+int launch_zero_pad_rows(void* q, void* k, void* v, int32_t q_row_bytes, int32_t kv_row_bytes,
+                         const int64_t* d_bin_used, int32_t n_bins, int32_t capacity, void* stream);
 
 int launch_bounded_wait_selftest(int32_t* device_status, uint64_t limit_ns, void* stream);
 

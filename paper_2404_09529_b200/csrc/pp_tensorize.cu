@@ -60,7 +60,38 @@ tensorize_kernel(uint4* __restrict__ packed, uint4* __restrict__ tokens, const i
   }
 }
 
+// Zeroes the padding rows [bin_used[b], capacity) of every bin of up to three packed tensors (the
+// attention kernels want finite values there); grid = (bins, row chunks).
+struct PadTensors {
+  uint4* base[3];
+  int32_t vec_per_row[3];
+};
+__global__ void __launch_bounds__(kTzThreads)
+zero_pad_rows_kernel(PadTensors t, const int64_t* __restrict__ bin_used, int32_t capacity) {
+  const int32_t b = blockIdx.x;
+  const int64_t used = bin_used[b];
+  const int64_t pad_rows = capacity - used;
+  for (int i = 0; i < 3; ++i) {
+    if (!t.base[i]) continue;
+    const int64_t n = pad_rows * t.vec_per_row[i];
+    uint4* dst = t.base[i] + ((int64_t)b * capacity + used) * t.vec_per_row[i];
+    for (int64_t u = (int64_t)blockIdx.y * kTzThreads + threadIdx.x; u < n; u += (int64_t)gridDim.y * kTzThreads)
+      dst[u] = make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
 }  // namespace
+
+int launch_zero_pad_rows(void* q, void* k, void* v, int32_t q_row_bytes, int32_t kv_row_bytes,
+                         const int64_t* d_bin_used, int32_t n_bins, int32_t capacity, void* stream) {
+  PadTensors t;
+  t.base[0] = static_cast<uint4*>(q); t.base[1] = static_cast<uint4*>(k); t.base[2] = static_cast<uint4*>(v);
+  t.vec_per_row[0] = q_row_bytes / 16; t.vec_per_row[1] = t.vec_per_row[2] = kv_row_bytes / 16;
+  zero_pad_rows_kernel<<<dim3((unsigned)n_bins, 8), kTzThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      t, d_bin_used, capacity);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? PP_OK : note_cuda_error((int)e, "padding-row kernel launch");
+}
 
 int launch_tensorize(bool to_packed, void* packed, void* tokens, const int64_t* d_map, int32_t n_prompts,
                      int64_t total_tokens, int32_t row_bytes, void* stream) {

@@ -20,8 +20,16 @@ class PrefillBatch:
     mask and tile skipping without the bin packing (isolates what packing adds).
     """
 
+    SENTINEL = -1.0e30      # bf16 value that pre-fills guard regions and cache pools (guard=True)
+
     def __init__(self, lengths, n_q_heads: int, n_kv_heads: int, head_dim: int, rope_base: float,
-                 mode: str = "packed", device: str = "cuda", softmax_scale: float = 0.0):
+                 mode: str = "packed", device: str = "cuda", softmax_scale: float = 0.0, room=0,
+                 guard: bool = False):
+        """room (int or one int per prompt): spare rows in every prompt's cache block, so that
+        cache_cap[i] = lengths[i] + room. guard: put sentinel-filled regions in front of and behind
+        every buffer the library writes (O, K, both cache pools) and pre-fill the pools with the
+        sentinel, so that `assert_untouched` can tell whether anything outside the documented
+        outputs was written."""
         self.device = torch.device(device)
         self.mode = mode
         self.lengths = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
@@ -32,22 +40,47 @@ class PrefillBatch:
         self._pack()
         R, M = self.pack.n_bins, self.pack.capacity
         dev, bf = self.device, torch.bfloat16
+        self._guards = []
         self.q = torch.zeros((R, M, n_q_heads, head_dim), dtype=bf, device=dev)
-        self.kk = torch.zeros((R, M, n_kv_heads, head_dim), dtype=bf, device=dev)
+        self.kk = self._alloc((R, M, n_kv_heads, head_dim), guard, 0.0)
         self.v = torch.zeros((R, M, n_kv_heads, head_dim), dtype=bf, device=dev)
-        self.o = torch.zeros((R, M, n_q_heads, head_dim), dtype=bf, device=dev)
-        # per-prompt caches, one pool each, [Hkv, l_i, D] blocks back to back in original order
-        self.cache_cap = self.lengths.copy()
-        tok_prefix = np.concatenate([[0], np.cumsum(self.lengths.astype(np.int64))])
-        self.cache_off = (tok_prefix[:-1] * n_kv_heads * head_dim).astype(np.int64)
-        pool = self.total_tokens * n_kv_heads * head_dim
-        self.k_cache = torch.zeros(pool, dtype=bf, device=dev)
-        self.v_cache = torch.zeros(pool, dtype=bf, device=dev)
+        self.o = self._alloc((R, M, n_q_heads, head_dim), guard, 0.0)
+        # per-prompt caches, one pool each, [Hkv, cap_i, D] blocks back to back in original order
+        self.cache_cap = (self.lengths + np.asarray(room, dtype=np.int32)).astype(np.int32)
+        cap_prefix = np.concatenate([[0], np.cumsum(self.cache_cap.astype(np.int64))])
+        self.cache_off = (cap_prefix[:-1] * n_kv_heads * head_dim).astype(np.int64)
+        pool = int(cap_prefix[-1]) * n_kv_heads * head_dim
+        self.k_cache = self._alloc((pool,), guard, self.SENTINEL if guard else 0.0)
+        self.v_cache = self._alloc((pool,), guard, self.SENTINEL if guard else 0.0)
         self.ws = B.Workspaces(self.params, self.pack.k, device=dev)
         # flat packed row of every real token, original prompt order
         rows = [np.arange(l, dtype=np.int64) + int(b) * M + int(off)
                 for l, b, off in zip(self.lengths, self.bin_of, self.off_of)]
         self.token_rows = torch.from_numpy(np.concatenate(rows)).to(dev)
+
+    def _alloc(self, shape, guard: bool, fill: float) -> torch.Tensor:
+        """A device tensor of `shape`; with guard, the middle of a larger sentinel-filled buffer."""
+        n = int(np.prod(shape))
+        if not guard:
+            return torch.full((n,), fill, dtype=torch.bfloat16, device=self.device).view(shape)
+        g = 4096                                          # elements: keeps the payload 8 KB aligned
+        whole = torch.full((n + 2 * g,), self.SENTINEL, dtype=torch.bfloat16, device=self.device)
+        self._guards.append((whole, g, n))
+        body = whole[g:g + n]
+        body.fill_(fill)
+        return body.view(shape)
+
+    def assert_untouched(self) -> None:
+        """Guard regions around O, K and the cache pools, and the spare rows [lengths[i], cap[i]) of
+        every cache block, still hold the sentinel bit for bit (needs guard=True)."""
+        assert self._guards, "PrefillBatch was built without guard=True"
+        for whole, g, n in self._guards:
+            for part in (whole[:g], whole[g + n:]):
+                assert bool((part == self.SENTINEL).all()), "write outside an output buffer"
+        for i in range(self.k):
+            l = int(self.lengths[i])
+            for c in self.caches(i):
+                assert bool((c[:, l:] == self.SENTINEL).all()), f"spare cache rows of prompt {i} were written"
 
     def _pack(self) -> None:
         """BINPACK through the library (host)."""
@@ -92,12 +125,17 @@ class PrefillBatch:
                            self.ws.unpack_bytes, stream)
         self.ws.release(slot)
 
-    def run_fused(self, repack: bool = False, flags: int = 0) -> None:
-        """One pass of the hot path through the fused entry point (asynchronous). q is left untouched."""
+    def run_fused(self, repack: bool = False, flags: int = 0, keep_rope_table: bool = True) -> None:
+        """One pass of the hot path through the fused entry point (asynchronous). q is left untouched.
+        The fused workspace is written by nothing but these calls, so from the second call with the
+        same capacity on, the cos/sin table in it is declared valid (PP_FLAG_KEEP_ROPE_TABLE)."""
         if repack:
             self._pack()
         stream = torch.cuda.current_stream().cuda_stream
         _, _, slot = self.ws.acquire()
+        if keep_rope_table and getattr(self, "_rope_table_capacity", None) == self.pack.capacity:
+            flags |= B.PP_FLAG_KEEP_ROPE_TABLE
+        self._rope_table_capacity = self.pack.capacity
         self.params.flags = flags
         B.pp_prefill_fused(self.params, self.pack, self.lengths, self.q, self.kk, self.v, self.o, self.k_cache,
                            self.v_cache, self.cache_off, self.cache_cap, self.ws.fused_dev,
@@ -126,8 +164,8 @@ class PrefillBatch:
                 self.kk.view(-1, self.hkv, self.d)[self.token_rows])
 
     def caches(self, i: int):
-        """(k_cache_i, v_cache_i) as [Hkv, l_i, D] views of the pools."""
-        n = int(self.lengths[i]) * self.hkv * self.d
+        """(k_cache_i, v_cache_i) as [Hkv, cap_i, D] views of the pools; rows [0, lengths[i]) are filled."""
+        n = int(self.cache_cap[i]) * self.hkv * self.d
         off = int(self.cache_off[i])
         shape = (self.hkv, int(self.cache_cap[i]), self.d)
         return self.k_cache[off:off + n].view(shape), self.v_cache[off:off + n].view(shape)
@@ -162,6 +200,23 @@ class DecodeBatch:
         off = int(self.cache_off[i])
         shape = (self.hkv, cap, self.d)
         return self.k_cache[off:off + n].view(shape), self.v_cache[off:off + n].view(shape)
+
+    @classmethod
+    def from_prefill(cls, prefill: PrefillBatch) -> "DecodeBatch":
+        """Decode straight on the cache pools a PrefillBatch (built with room > 0) has filled: the
+        hand-over from UNPACK to generation, no copy in between."""
+        self = cls.__new__(cls)
+        self.device = prefill.device
+        self.lengths = prefill.lengths.copy()
+        self.k = prefill.k
+        self.hq, self.hkv, self.d = prefill.hq, prefill.hkv, prefill.d
+        self.cache_cap, self.cache_off = prefill.cache_cap, prefill.cache_off
+        self.k_cache, self.v_cache = prefill.k_cache, prefill.v_cache
+        self.params = B.AttnParams(self.hq, self.hkv, self.d, prefill.rope_base, prefill.softmax_scale, 1, 1, 0)
+        self.o = torch.zeros((self.k, self.hq, self.d), dtype=torch.bfloat16, device=self.device)
+        self._ws_bytes = 0
+        self._ws = self._host = None
+        return self
 
     def adopt(self, prefill: PrefillBatch) -> None:
         for i in range(self.k):

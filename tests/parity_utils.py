@@ -38,12 +38,14 @@ class ErrStat:
         assert self.mean_abs <= MEAN_ABS_TOL, (what, "mean", self.mean_abs)
 
 
-def run_cuda(lengths, q_tok, k_tok, v_tok, hq, hkv, d, base, mode="packed"):
-    batch = PrefillBatch(lengths, hq, hkv, d, base, mode=mode)
+def run_cuda(lengths, q_tok, k_tok, v_tok, hq, hkv, d, base, mode="packed", fused=False, room=0, guard=False):
+    batch = PrefillBatch(lengths, hq, hkv, d, base, mode=mode, room=room, guard=guard)
     batch.load(q_tok, k_tok, v_tok)
-    batch.run()
+    batch.run_fused() if fused else batch.run()
     torch.cuda.synchronize()
     assert batch.device_status() == 0
+    if guard:
+        batch.assert_untouched()
     return batch
 
 
@@ -55,12 +57,58 @@ def compare_full(batch, lengths, q_tok, k_tok, v_tok, base, prompts=None):
     for i in (range(len(lengths)) if prompts is None else prompts):
         o_ref, kc_ref, vc_ref = orc.prefill_prompt(to64(qs[i]), to64(ks[i]), to64(vs[i]), base)
         kc, vc = batch.caches(i)
+        l = int(lengths[i])                       # a cache block may have spare rows behind the prompt
         e_o.add(to64(o_cuda[i]), o_ref)
-        e_k.add(to64(kc), kc_ref)
-        e_v.add(to64(vc), vc_ref)
+        e_k.add(to64(kc[:, :l]), kc_ref)
+        e_v.add(to64(vc[:, :l]), vc_ref)
     e_o.check("O"); e_k.check("K cache"); e_v.check("V cache")
     assert e_v.max_abs == 0.0
     return e_o, e_k, e_v
+
+
+def oracle_refs(lengths, q_tok, k_tok, v_tok, base):
+    """The oracle's (O, K cache, V cache) of every prompt alone, computed once for several runs."""
+    qs, ks, vs = (split_by_prompt(t.cpu(), lengths) for t in (q_tok, k_tok, v_tok))
+    return [orc.prefill_prompt(to64(qs[i]), to64(ks[i]), to64(vs[i]), base) for i in range(len(lengths))]
+
+
+def compare_with_refs(batch, lengths, refs):
+    """Every row, head and cache element of every prompt against precomputed oracle results."""
+    o_cuda = split_by_prompt(batch.o_tokens().cpu(), lengths)
+    e_o, e_k, e_v = ErrStat(), ErrStat(), ErrStat()
+    for i, (o_ref, kc_ref, vc_ref) in enumerate(refs):
+        kc, vc = batch.caches(i)
+        l = int(lengths[i])
+        e_o.add(to64(o_cuda[i]), o_ref)
+        e_k.add(to64(kc[:, :l]), kc_ref)
+        e_v.add(to64(vc[:, :l]), vc_ref)
+    e_o.check("O"); e_k.check("K cache"); e_v.check("V cache")
+    assert e_v.max_abs == 0.0
+    return e_o, e_k, e_v
+
+
+def expected_schedule(seg_bins, hq, hkv):
+    """What the attention kernel's host scheduler must choose for a packing, restated from its rule
+    (independent of the library): seg_bins is a list of bins, each a list of segment lengths in
+    placement order. Mean number of 128-row key tiles per 128-row query tile, counting for a query
+    tile the key rows from the 128-aligned start of the first prompt it touches to its last row:
+    below 8 the kernel runs its independent mode (64-row key tiles, template <D, true>), otherwise
+    its shared-stream mode (template <D, false>), pairing two query heads when the GQA group is even
+    and two consecutive row tiles otherwise. Returns (mode, pairing) as pp_prefill_schedule_info
+    numbers them."""
+    q_tiles = kv_tiles = 0
+    for segs in seg_bins:
+        starts = np.concatenate([[0], np.cumsum(segs)])
+        used = int(starts[-1])
+        for q0 in range(0, used, 128):
+            s = int(np.searchsorted(starts[:-1], q0, side="right")) - 1
+            kv_lo = (int(starts[s]) // 128) * 128
+            kv_tiles += (min(q0 + 128, used) - kv_lo + 127) // 128
+            q_tiles += 1
+    independent = kv_tiles / q_tiles < 8.0
+    if independent:
+        return 1, 2
+    return 0, (0 if (hq // hkv) % 2 == 0 else 1)
 
 
 def compare_sampled(batch, lengths, q_tok, k_tok, v_tok, base, prompts, kv_heads, n_rows, seed=0):
@@ -82,8 +130,8 @@ def compare_sampled(batch, lengths, q_tok, k_tok, v_tok, base, prompts, kv_heads
         o_ref, kc_ref, vc_ref = orc.prefill_prompt(q, k, v, base, rows=rows)
         e_o.add(to64(o_all[sl][rows][:, q_heads]), o_ref)
         kc, vc = batch.caches(i)
-        e_k.add(to64(kc[kv_heads]), kc_ref)
-        e_v.add(to64(vc[kv_heads]), vc_ref)
+        e_k.add(to64(kc[kv_heads][:, :l]), kc_ref)
+        e_v.add(to64(vc[kv_heads][:, :l]), vc_ref)
     e_o.check("O"); e_k.check("K cache"); e_v.check("V cache")
     assert e_v.max_abs == 0.0
     return e_o, e_k, e_v

@@ -165,7 +165,7 @@ def test_host_buffer_entry_point_matches_device_path():
 
 
 @pytest.mark.parametrize("groups", [1, 3, 8])
-def test_host_buffer_entry_point_pipelined_groups(groups, monkeypatch):
+def test_host_buffer_entry_point_pipelined_groups(groups):
     """pp_prefill_host cuts large batches into groups of prompts, each packed on its own and run on
     its own stream. Caches do not depend on the packing (bit-identical to the whole-batch run); O
     depends on it only through the position of tile boundaries (summation order)."""
@@ -174,7 +174,7 @@ def test_host_buffer_entry_point_pipelined_groups(groups, monkeypatch):
     hq, hkv, d, base = 8, 2, 128, 500000.0
     q, k, v = _random_case(lengths, hq, hkv, d, seed=5)
     ref = run_cuda(lengths, q, k, v, hq, hkv, d, base)
-    monkeypatch.setenv("PP_HOST_GROUPS", str(groups))
+    before = pp.pp_prefill_host_groups(groups)
     params = pp.AttnParams(hq, hkv, d, base, 0.0, 0, 0, 0)
     nbytes = pp.pp_prefill_host_arena_bytes(params, lengths)
     arena = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
@@ -193,6 +193,7 @@ def test_host_buffer_entry_point_pipelined_groups(groups, monkeypatch):
         else:
             diff = (o.float() - ref.o_tokens().cpu().float()).abs()
             assert float(diff.max()) <= 2e-2 and float(diff.mean()) <= 5e-4
+    assert pp.pp_prefill_host_groups(before) == groups
 
 
 def test_bounded_wait_gives_up_and_reports():

@@ -128,6 +128,10 @@ def test_prefill_argument_validation_happens_before_any_device_work():
     bad.seg_start[2] = 80                             # gap inside a bin
     assert call(_params(), pack=bad) == -1
     assert pp.pp_prefill_workspace_bytes(_params(head_dim=32), 8) == 0
+    # flag bits the header does not define (two of them were internal options once) are refused
+    for bad in (0x100, 0x200, 0x8, 1 << 30):
+        assert call(_params(flags=bad)) == -1
+        assert call(_params(flags=bad | pp.PP_FLAG_SKIP_ROPE)) == -1
 
 
 def test_unpack_argument_validation():
@@ -151,3 +155,66 @@ def test_unpack_argument_validation():
     assert call(kc=A + 2) == -5
     assert call(wb=ws - 1) == -3
     assert call(cache_cap=(4, 10)) == -2
+
+
+def test_schedule_info_matches_the_scheduling_rule():
+    """pp_prefill_schedule_info (host only) against the rule restated in the test helpers, on packings
+    around the mode threshold and with odd / even GQA groups."""
+    import sys, os
+    sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+    from parity_utils import expected_schedule
+    rng = np.random.default_rng(7)
+    for trial in range(60):
+        kind = trial % 3
+        if kind == 0:
+            lengths = rng.integers(1, 400, size=int(rng.integers(1, 40)))
+        elif kind == 1:
+            lengths = rng.integers(600, 4000, size=int(rng.integers(1, 6)))
+        else:
+            lengths = np.concatenate([rng.integers(900, 1400, size=3), rng.integers(1, 50, size=int(rng.integers(0, 30)))])
+        hkv = int(rng.choice([1, 2]))
+        hq = hkv * int(rng.choice([1, 2, 3, 4]))
+        pk = pp.pp_pack(lengths)
+        info = pp.pp_prefill_schedule_info(_params(n_q_heads=hq, n_kv_heads=hkv, capacity=pk.capacity, n_bins=pk.n_bins), pk)
+        seg_bins = [[int(x) for x in pk.seg_len[pk.bin_seg_ptr[b]:pk.bin_seg_ptr[b + 1]]] for b in range(pk.n_bins)]
+        assert (info["mode"], info["pairing"]) == expected_schedule(seg_bins, hq, hkv), (lengths, hq, hkv, info)
+        assert info["key_tile_rows"] == (64 if info["mode"] == 1 else 128)
+        assert info["entries"] >= pk.n_bins and info["steps"] >= info["entries"]
+
+
+def test_per_device_once_guard(tmp_path):
+    """The record that keeps per-device kernel set-up from running twice (and, above all, from being
+    skipped on a second GPU): compiled on its own with the host compiler and driven from two threads."""
+    import shutil, subprocess, textwrap
+    gxx = shutil.which("g++")
+    if gxx is None:
+        pytest.skip("no host C++ compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "once.cpp"
+    src.write_text(textwrap.dedent("""
+        #include "pp_device_once.h"
+        #include <cstdio>
+        #include <thread>
+        int main() {
+          pp::DeviceOnce once;
+          for (int d = -2; d < 200; ++d) if (once.done(d)) return 1;          // nothing done at start
+          once.mark(0);
+          if (!once.done(0) || once.done(1) || once.done(63) || once.done(64)) return 2;   // per device
+          once.mark(64); once.mark(127);
+          if (!once.done(64) || !once.done(127) || once.done(65) || once.done(126)) return 3;
+          once.mark(-1); once.mark(128); once.mark(1000);                      // out of range: never recorded
+          if (once.done(-1) || once.done(128) || once.done(1000)) return 4;
+          pp::DeviceOnce shared;
+          std::thread a([&] { for (int d = 0; d < 128; d += 2) shared.mark(d); });
+          std::thread b([&] { for (int d = 1; d < 128; d += 2) shared.mark(d); });
+          a.join(); b.join();
+          for (int d = 0; d < 128; ++d) if (!shared.done(d)) return 5;         // no lost update
+          std::puts("ok");
+          return 0;
+        }
+    """))
+    exe = tmp_path / "once"
+    inc = os.path.join(root, "paper_2404_09529_b200", "csrc")
+    subprocess.run([gxx, "-std=c++17", "-O1", "-pthread", "-I", inc, str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0 and out.stdout.strip() == "ok", (out.returncode, out.stdout, out.stderr)
