@@ -39,7 +39,7 @@ def test_own_arm_line():
     assert d["n_gpus"] == 1 and d["steps"] == 3 and d["warmup"] == 3 and d["higher_is_better"] is True
     assert d["scaling"] == "weak" and d["vs_baseline"] is None and d["data"] == "synthetic"
     assert d["config"]["workload"] == "tiny" and "model" not in d["config"]
-    assert d["gpu_launches"] == 3 * d["steps"]
+    assert d["gpu_launches"] == 2 * d["steps"]
     r = d["roofline"]
     assert {"bound", "achieved", "peak", "unit", "frac", "traffic"} <= set(r) and r["bound"] in ("hbm", "tensor", "alu")
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
