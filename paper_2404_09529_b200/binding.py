@@ -136,6 +136,18 @@ class Packing:
     def k(self) -> int:
         return int(self.seg_start.shape[0])
 
+    def slice_bins(self, b0: int, b1: int):
+        """Bins [b0, b1) as a packing of their own (index bookkeeping only). Returns (packing, prompts):
+        `prompts` are the original indices of the prompts in those bins, ascending, and the packing's
+        seg_prompt / bin_of / off_of refer to positions in that list."""
+        s0, s1 = int(self.bin_seg_ptr[b0]), int(self.bin_seg_ptr[b1])
+        seg_prompt = self.seg_prompt[s0:s1]
+        prompts = np.sort(seg_prompt)
+        local = np.searchsorted(prompts, seg_prompt).astype(np.int32)
+        return (Packing(b1 - b0, self.capacity, (self.bin_seg_ptr[b0:b1 + 1] - s0).astype(np.int32), local,
+                        self.seg_start[s0:s1].copy(), self.seg_len[s0:s1].copy(),
+                        (self.bin_of[prompts] - b0).astype(np.int32), self.off_of[prompts].copy()), prompts)
+
 
 def pp_pack(lengths, capacity: int = 0) -> Packing:
     lib = load_library()

@@ -262,6 +262,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// Bits [c_lo, c_hi] of a 64-bit word set (none if the interval is empty); c_hi <= 63, c_lo >= 0.
+__device__ __forceinline__ uint64_t visible_mask64(int c_lo, int c_hi) {
+  if (c_hi < c_lo) return 0ull;
+  return (~0ull << c_lo) & (~0ull >> (63 - c_hi));
+}
+
 // Instruction descriptor: fp32 accumulate, bf16 A and B, A K-major, M = 128.
 __host__ __device__ constexpr uint32_t instr_desc(uint32_t n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) |
@@ -808,11 +814,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // one warp reduction for all the per-warp flags of the tile: which 32-column chunks
             // somebody can see, and whether any row's interval ends or begins inside the tile
             static_assert(NCH == 2, "flag bits below are laid out for two chunks");
-            const uint32_t lane_flags = (uint32_t)(c_lo <= min(c_hi, 31)) | ((uint32_t)(max(c_lo, 32) <= c_hi) << 1) |
-                                        ((uint32_t)(c_hi < EPT - 1) << 2) | ((uint32_t)(c_lo > 0) << 3);
+            const uint64_t vis = visible_mask64(c_lo, c_hi);     // bit i: column i is visible to this row
+            const uint32_t vis_lo = (uint32_t)vis, vis_hi = (uint32_t)(vis >> 32);
+            const uint32_t lane_flags = (uint32_t)(vis_lo != 0u) | ((uint32_t)(vis_hi != 0u) << 1) |
+                                        ((uint32_t)(~vis != 0ull) << 2);
             const uint32_t warp_flags = __reduce_or_sync(0xffffffffu, lane_flags);
             const bool need[NCH] = {(warp_flags & 1u) != 0, (warp_flags & 2u) != 0};
-            const bool cut_hi = (warp_flags & 4u) != 0, cut_lo = (warp_flags & 8u) != 0;
+            const bool cut = (warp_flags & 4u) != 0;
             const uint32_t sbuf = tcount & 1u;                   // tile k of the stream lives in S buffer k & 1
             const uint32_t tmem_sb = tmem_s + 64u * sbuf;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * (2 * t + sbuf), (tcount >> 1) & 1u, wctx, kWaitS));
@@ -829,15 +837,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               }
             }
             tc_wait_ld();
-            // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
-            // one of the two bounds (the causal diagonal, or the first tile of a prompt)
-            if (cut_hi) {
+            // masked tiles (the causal diagonal, the first tile of a prompt): one select per score,
+            // steered by the bits of the row's visibility mask
+            if (cut) {
 #pragma unroll
-              for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
-            }
-            if (cut_lo) {
+              for (int i = 0; i < 32; ++i) v[i] = (vis_lo & (1u << i)) ? v[i] : 0xff800000u;
 #pragma unroll
-              for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
+              for (int i = 0; i < 32; ++i) v[32 + i] = (vis_hi & (1u << i)) ? v[32 + i] : 0xff800000u;
             }
             float mx;
             {
@@ -1142,11 +1148,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // one warp reduction for all the per-warp flags of the tile: which 32-column chunks somebody
         // can see, and whether any row's interval ends or begins inside this half of the tile
         static_assert(NCH == 2, "flag bits below are laid out for two chunks");
-        const uint32_t lane_flags = (uint32_t)(c_lo <= min(c_hi, 31)) | ((uint32_t)(max(c_lo, 32) <= c_hi) << 1) |
-                                    ((uint32_t)(c_hi < EPT - 1) << 2) | ((uint32_t)(c_lo > 0) << 3);
+        const uint64_t vis = visible_mask64(c_lo, c_hi);     // bit i: column i is visible to this row
+        const uint32_t vis_lo = (uint32_t)vis, vis_hi = (uint32_t)(vis >> 32);
+        const uint32_t lane_flags = (uint32_t)(vis_lo != 0u) | ((uint32_t)(vis_hi != 0u) << 1) |
+                            ((uint32_t)(~vis != 0ull) << 2);
         const uint32_t warp_flags = __reduce_or_sync(0xffffffffu, lane_flags);
         const bool need[NCH] = {(warp_flags & 1u) != 0, (warp_flags & 2u) != 0};
-        const bool cut_hi = (warp_flags & 4u) != 0, cut_lo = (warp_flags & 8u) != 0;
+        const bool cut = (warp_flags & 4u) != 0;
         const uint32_t sbuf = 0u;
         const uint32_t tparity = tcount & 1u;
         const uint32_t tmem_sb = tmem_s;
@@ -1166,15 +1174,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         tc_wait_ld();
-        // the visible columns of a row are one interval [c_lo, c_hi]; most masked tiles need only
-        // one of the two bounds (the causal diagonal, or the first tile of a prompt)
-        if (cut_hi) {
+        // masked tiles (the causal diagonal, the first tile of a prompt): one select per score,
+        // steered by the bits of the row's visibility mask
+        if (cut) {
 #pragma unroll
-          for (int i = 0; i < EPT; ++i) v[i] = (i <= c_hi) ? v[i] : 0xff800000u;
-        }
-        if (cut_lo) {
+          for (int i = 0; i < 32; ++i) v[i] = (vis_lo & (1u << i)) ? v[i] : 0xff800000u;
 #pragma unroll
-          for (int i = 0; i < EPT; ++i) v[i] = (i >= c_lo) ? v[i] : 0xff800000u;
+          for (int i = 0; i < 32; ++i) v[32 + i] = (vis_hi & (1u << i)) ? v[32 + i] : 0xff800000u;
         }
         float mx;
         {

@@ -24,14 +24,16 @@ class PrefillBatch:
 
     def __init__(self, lengths, n_q_heads: int, n_kv_heads: int, head_dim: int, rope_base: float,
                  mode: str = "packed", device: str = "cuda", softmax_scale: float = 0.0, room=0,
-                 guard: bool = False):
+                 guard: bool = False, pack: "B.Packing | None" = None):
         """room (int or one int per prompt): spare rows in every prompt's cache block, so that
         cache_cap[i] = lengths[i] + room. guard: put sentinel-filled regions in front of and behind
         every buffer the library writes (O, K, both cache pools) and pre-fill the pools with the
         sentinel, so that `assert_untouched` can tell whether anything outside the documented
-        outputs was written."""
+        outputs was written. pack: a packing made elsewhere (e.g. some bins of a packing of a whole
+        stream of prompts, Packing.slice_bins) for exactly these prompts; mode is then "prepacked"."""
         self.device = torch.device(device)
-        self.mode = mode
+        self.mode = "prepacked" if pack is not None else mode
+        self._given_pack = pack
         self.lengths = np.ascontiguousarray(np.asarray(lengths, dtype=np.int32))
         self.k = int(self.lengths.shape[0])
         self.total_tokens = int(self.lengths.sum())
@@ -84,7 +86,10 @@ class PrefillBatch:
 
     def _pack(self) -> None:
         """BINPACK through the library (host)."""
-        if self.mode == "packed":
+        if self.mode == "prepacked":
+            self.pack = self._given_pack
+            self.bin_of, self.off_of = self.pack.bin_of, self.pack.off_of
+        elif self.mode == "packed":
             self.pack = B.pp_pack(self.lengths, 0)
             self.bin_of, self.off_of = self.pack.bin_of, self.pack.off_of
         elif self.mode == "padded":

@@ -5,8 +5,8 @@ and the padded (full-batching) path are timed and the speedup is regressed on th
 statistics the paper uses: the bin reduction r / k and the padding per prompt m - L / k
 (m = longest prompt, L = total tokens, r = bins after packing). Attention layer only.
 
-``dataset``: a stream of prompts is prefilled (a) prepacked as a whole and processed in launches
-of a fixed number of bins, (b) in batches of consecutive prompts after sorting the stream by
+``dataset``: a stream of prompts is prefilled (a) bin-packed as a whole, once, and processed in
+launches of a fixed number of bins of that one packing, (b) in batches of consecutive prompts after sorting the stream by
 length, each padded to its own maximum, (c) in batches in arrival order, padded. Reports useful
 tokens per second of each schedule.
 
@@ -30,6 +30,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import time
 
 import numpy as np
 import torch
@@ -58,26 +59,27 @@ def _time_ms(fn, iters: int = 5, warmup: int = 2) -> float:
     return e0.elapsed_time(e1) / iters
 
 
-def _batch(lengths: np.ndarray, mode: str, gen: torch.Generator) -> PrefillBatch:
-    b = PrefillBatch(lengths, HQ, HKV, D, BASE, mode=mode)
-    t = int(lengths.sum())
-    q = torch.randn(t, HQ, D, generator=gen, device="cuda").to(torch.bfloat16)
-    k = torch.randn(t, HKV, D, generator=gen, device="cuda").to(torch.bfloat16)
-    v = torch.randn(t, HKV, D, generator=gen, device="cuda").to(torch.bfloat16)
-    b.load(q, k, v)
-    return b
-
-
-def predictor(n_batches: int, k: int, seed: int) -> dict:
+def predictor(n_batches: int, k: int, seed: int, probe=None) -> dict:
+    """`probe(packed_batch, padded_batch, q, k, v, lengths)`, if given, is called with the first batch
+    after both paths have run on the same tensors (tests check the outputs)."""
     rng = np.random.default_rng(seed)
     gen = torch.Generator(device="cuda").manual_seed(seed)
     rows = []
-    for _ in range(n_batches):
+    for i in range(n_batches):
         lengths = rng.integers(1, 513, size=k).astype(np.int32)
-        packed, padded = _batch(lengths, "packed", gen), _batch(lengths, "padded", gen)
+        t = int(lengths.sum())
+        tensors = tuple(torch.randn(t, h, D, generator=gen, device="cuda").to(torch.bfloat16) for h in (HQ, HKV, HKV))
+        packed = PrefillBatch(lengths, HQ, HKV, D, BASE, mode="packed")
+        padded = PrefillBatch(lengths, HQ, HKV, D, BASE, mode="padded")
+        packed.load(*tensors); padded.load(*tensors)
         ms_packed = _time_ms(lambda: packed.run_fused(repack=True))
         ms_padded = _time_ms(lambda: padded.run_fused(repack=True))
         assert packed.device_status() == 0 and padded.device_status() == 0
+        if probe is not None and i == 0:
+            packed.load(*tensors); padded.load(*tensors)
+            packed.run_fused(); padded.run_fused()
+            torch.cuda.synchronize()
+            probe(packed, padded, *tensors, lengths)
         m, total, r = int(lengths.max()), int(lengths.sum()), int(packed.pack.n_bins)
         rows.append({"r_over_k": r / k, "pad_per_prompt": m - total / k, "speedup": ms_padded / ms_packed,
                      "ms_packed": ms_packed, "ms_padded": ms_padded})
@@ -95,36 +97,71 @@ def predictor(n_batches: int, k: int, seed: int) -> dict:
             "rows": rows}
 
 
-def dataset(n_prompts: int, batch: int, seed: int) -> dict:
+def dataset(n_prompts: int, batch: int, seed: int, bins_per_launch: int = 0, probe=None) -> dict:
+    """Section 6: the whole stream of prompts is bin-packed once (pp_pack, bin size = the longest prompt
+    of the stream), the bins are then processed `bins_per_launch` at a time (default: the bin count a
+    launch of `batch` * 16 average prompts fills), each launch through pp_prefill_fused on its slice of
+    the one packing. Compared on the same stream with length-ordered batching (sort, padded batches of
+    `batch`) and with padded batches in arrival order. `probe(batch, q, k, v, lengths)`, if given, is
+    called once with a finished launch of every schedule (tests check its outputs)."""
+    from . import binding as B
     rng = np.random.default_rng(seed)
     gen = torch.Generator(device="cuda").manual_seed(seed)
     lengths = np.clip(np.rint(np.exp(np.log(200.0) + 0.8 * rng.standard_normal(n_prompts))), 8, 2048).astype(np.int32)
     total = int(lengths.sum())
 
-    def run_schedule(groups, mode):
-        ms = 0.0
-        for g in groups:
-            b = _batch(g, mode, gen)
-            ms += _time_ms(lambda: b.run_fused(repack=True), iters=3, warmup=1)
-            assert b.device_status() == 0
-            del b
+    def qkv(ls):
+        t = int(ls.sum())
+        return tuple(torch.randn(t, h, D, generator=gen, device="cuda").to(torch.bfloat16) for h in (HQ, HKV, HKV))
+
+    def run_launch(b, tensors, ls, repack, probed):
+        b.load(*tensors)
+        ms = _time_ms(lambda: b.run_fused(repack=repack), iters=3, warmup=1)
+        assert b.device_status() == 0
+        if probe is not None and not probed:
+            b.load(*tensors)
+            b.run_fused(repack=repack)
+            torch.cuda.synchronize()
+            probe(b, *tensors, ls)
         return ms
 
-    # (a) prepack the whole stream, launches of `batch` prompts' worth of tokens each: the packer is
-    # run per launch group of consecutive prompts large enough to fill many bins
-    per_launch = batch * 16
-    packed_groups = [lengths[i:i + per_launch] for i in range(0, n_prompts, per_launch)]
-    ms_prepacked = run_schedule(packed_groups, "packed")
+    # (a) one packing of the whole stream, launches of consecutive bins
+    t0 = time.perf_counter()
+    whole = B.pp_pack(lengths, 0)
+    pack_ms = (time.perf_counter() - t0) * 1e3
+    if bins_per_launch <= 0:
+        bins_per_launch = max(1, int(round(batch * 16 * float(lengths.mean()) / whole.capacity)))
+    ms_prepacked, launches = 0.0, 0
+    for b0 in range(0, whole.n_bins, bins_per_launch):
+        b1 = min(b0 + bins_per_launch, whole.n_bins)
+        part, prompts = whole.slice_bins(b0, b1)
+        ls = lengths[prompts]
+        bt = PrefillBatch(ls, HQ, HKV, D, BASE, pack=part)
+        ms_prepacked += run_launch(bt, qkv(ls), ls, False, launches > 0)
+        launches += 1
+        del bt
+
+    def run_padded(groups):
+        ms = 0.0
+        for i, g in enumerate(groups):
+            bt = PrefillBatch(g, HQ, HKV, D, BASE, mode="padded")
+            ms += run_launch(bt, qkv(g), g, True, i > 0)
+            del bt
+        return ms
+
     # (b) length-ordered batching: sort, then padded batches of `batch`
     order = np.sort(lengths)
-    ms_sorted = run_schedule([order[i:i + batch] for i in range(0, n_prompts, batch)], "padded")
+    ms_sorted = run_padded([order[i:i + batch] for i in range(0, n_prompts, batch)])
     # (c) arrival order, padded batches of `batch`
-    ms_arrival = run_schedule([lengths[i:i + batch] for i in range(0, n_prompts, batch)], "padded")
+    ms_arrival = run_padded([lengths[i:i + batch] for i in range(0, n_prompts, batch)])
     tps = lambda ms: total / (ms * 1e-3)
     return {"sweep": "dataset", "prompts": n_prompts, "total_tokens": total,
             "lengths": "lognormal(median 200, sigma 0.8) clipped to [8, 2048]",
             "layer": {"n_q_heads": HQ, "n_kv_heads": HKV, "head_dim": D},
-            "prepacked": {"prompts_per_launch": per_launch, "ms": ms_prepacked, "tokens_per_s": tps(ms_prepacked)},
+            "prepacked": {"bins": int(whole.n_bins), "capacity": int(whole.capacity), "bins_per_launch": bins_per_launch,
+                          "launches": launches, "pack_ms_host": pack_ms, "ms": ms_prepacked,
+                          "tokens_per_s": tps(ms_prepacked),
+                          "fill": total / (int(whole.n_bins) * int(whole.capacity))},
             "length_ordered_padded": {"batch": batch, "ms": ms_sorted, "tokens_per_s": tps(ms_sorted)},
             "arrival_order_padded": {"batch": batch, "ms": ms_arrival, "tokens_per_s": tps(ms_arrival)},
             "speedup_vs_arrival_order": ms_arrival / ms_prepacked,

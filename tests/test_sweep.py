@@ -1,12 +1,29 @@
-"""The measurement sweeps run end to end on small inputs (GPU only: the library has no CPU path)."""
+"""The measurement sweeps run end to end on small inputs (GPU only: the library has no CPU path), and
+one batch of each is checked against the float64 oracle: every row, head and cache element of its
+longest and its shortest prompt."""
+import numpy as np
 import pytest
 
 pytestmark = pytest.mark.gpu
 
 
+def _check_against_oracle(batch, q, k, v, lengths):
+    from parity_utils import compare_full
+    order = np.argsort(lengths)
+    compare_full(batch, np.asarray(lengths), q, k, v, batch.rope_base, prompts=sorted({int(order[0]), int(order[-1])}))
+
+
 def test_predictor_sweep_small():
     from paper_2404_09529_b200 import sweep
-    out = sweep.predictor(n_batches=4, k=8, seed=1)
+    seen = []
+
+    def probe(packed, padded, q, k, v, lengths):
+        _check_against_oracle(packed, q, k, v, lengths)
+        _check_against_oracle(padded, q, k, v, lengths)
+        seen.append(len(lengths))
+
+    out = sweep.predictor(n_batches=4, k=8, seed=1, probe=probe)
+    assert seen == [8]
     assert out["batches"] == 4 and len(out["rows"]) == 4
     for row in out["rows"]:
         assert 0.0 < row["r_over_k"] <= 1.0 and row["pad_per_prompt"] >= 0.0
@@ -16,8 +33,19 @@ def test_predictor_sweep_small():
 
 def test_dataset_sweep_small():
     from paper_2404_09529_b200 import sweep
-    out = sweep.dataset(n_prompts=64, batch=8, seed=1)
+    seen = []
+
+    def probe(batch, q, k, v, lengths):
+        _check_against_oracle(batch, q, k, v, lengths)
+        seen.append(batch.mode)
+
+    out = sweep.dataset(n_prompts=64, batch=8, seed=1, bins_per_launch=3, probe=probe)
+    assert seen == ["prepacked", "padded", "padded"]
     assert out["total_tokens"] > 0
+    # one packing of the whole stream: bins of the stream-wide capacity, cut into launches of 3 bins
+    pre = out["prepacked"]
+    assert pre["launches"] == -(-pre["bins"] // 3) and pre["launches"] > 1
+    assert pre["bins"] * pre["capacity"] >= out["total_tokens"] and 0.5 < pre["fill"] <= 1.0
     for key in ("prepacked", "length_ordered_padded", "arrival_order_padded"):
         assert out[key]["tokens_per_s"] > 0.0
     # with a lognormal length mix, padding to the batch maximum in arrival order wastes the most
