@@ -65,7 +65,8 @@ extern "C" const char* pp_last_cuda_error(void) { return pp::g_cuda_error; }
 
 extern "C" size_t pp_prefill_workspace_bytes(const pp_attn_params* params, int32_t k) {
   if (pp::check_params(params) != PP_OK || k < 1) return 0;
-  return sizeof(int32_t) * pp::prefill_table_ints(params->n_bins, params->capacity, k);
+  return sizeof(int32_t) * pp::prefill_table_ints(params->n_bins, params->capacity, k,
+                                                  params->n_q_heads / params->n_kv_heads);
 }
 
 extern "C" int pp_prefill_attention(const pp_attn_params* params, const int32_t* bin_seg_ptr,
@@ -125,7 +126,7 @@ struct FusedLayout {
 FusedLayout fused_layout(const pp_attn_params& p, int32_t k) {
   auto up4 = [](size_t x) { return (x + 3) & ~size_t(3); };
   FusedLayout f;
-  f.table_ints = prefill_table_ints(p.n_bins, p.capacity, k);
+  f.table_ints = prefill_table_ints(p.n_bins, p.capacity, k, p.n_q_heads / p.n_kv_heads);
   f.off_true_len = up4(f.table_ints);
   f.off_cap = f.off_true_len + up4((size_t)k);
   f.off_cache_off = f.off_cap + up4((size_t)k);          // multiple of 4 ints: 16-byte aligned int64 data

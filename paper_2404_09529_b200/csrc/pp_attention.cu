@@ -21,6 +21,11 @@
 // Independent mode (short items). Every slot draws its own items (one query tile each) and walks
 // their 64-row key tiles on its own; S_t has two 64-column buffers so that the scores of tile k+1
 // and the product P(k) V(k) are computed while the softmax threads work on tile k.
+// With several query heads per KV head (GQA) the heads are folded into the rows of a query tile:
+// 128 / f bin rows x f heads (tile row m = bin row m / f, head m % f; f = 2, 4 or 8 dividing the
+// group), loaded and stored as one TMA box over (row, head). One stream of key tiles then serves
+// the f heads, a short prompt fills a tile with heads instead of empty rows, and an item's key
+// tiles start at the first row of the first prompt it touches rather than at a tile boundary.
 //   warps 0-1    issue the tcgen05.mma of slot 0 / slot 1
 //   warps 2-3    draw items and TMA-load Q, K, V of slot 0 / slot 1 (two K and two V stages each)
 //   warps 4-7    softmax threads of slot 0, one per query row; they never leave the tile loop
@@ -282,6 +287,8 @@ struct AttnArgs {
   int32_t subs;                  // work indices per (KV head, geometry entry)
   int32_t pair_heads;            // 1: slots are two query heads; 0: two row tiles of one head
   int32_t group;                 // query heads per KV head
+  int32_t fold;                  // independent mode: query heads folded into a query tile (tile row m is
+  int32_t fold_shift;            //   bin row q_row0 + (m >> fold_shift) of head head[0] + (m & (fold - 1)))
   int32_t n_q_heads;
   int32_t capacity;              // rows per bin
   int32_t total_work;            // n_kv_heads * n_items * subs
@@ -313,7 +320,7 @@ __device__ __forceinline__ void decode_work(const AttnArgs& a, int w, Work& wk) 
     wk.head[0] = wk.kv_head * a.group + 2 * sub;
     wk.head[1] = wk.head[0] + 1;
   } else {
-    wk.head[0] = wk.head[1] = wk.kv_head * a.group + sub;
+    wk.head[0] = wk.head[1] = wk.kv_head * a.group + sub * a.fold;
   }
 }
 
@@ -341,10 +348,11 @@ enum WaitCode { kWaitItemFull = 1, kWaitItemEmpty, kWaitQFull, kWaitQEmpty, kWai
 
 // Start row of the prompt that holds bin-local row `i_row`, among the prompts seg_begin .. seg_end-1
 // of a bin whose start rows (ascending) are in `starts`; `lo` if none of them starts at or before the
-// row. All 32 lanes call it with the same range: the starts are loaded 32 at a time, one per lane,
-// and handed round with shuffles, so the walk costs one memory round trip per 32 prompts.
-__device__ __forceinline__ int seg_start_at(const int32_t* starts, int seg_begin, int seg_end, int i_row, int lo, int lane) {
-  const int row_max = i_row - lane + 31;               // the warp's rows are consecutive
+// row. All 32 lanes call it with the same range and with row_max = the largest row of the warp: the
+// starts are loaded 32 at a time, one per lane, and handed round with shuffles, so the walk costs one
+// memory round trip per 32 prompts.
+__device__ __forceinline__ int seg_start_at(const int32_t* starts, int seg_begin, int seg_end, int i_row, int row_max,
+                                            int lo, int lane) {
   for (int base = seg_begin; base < seg_end; base += 32) {
     const int cnt = min(32, seg_end - base);
     const int mine = (lane < cnt) ? __ldg(starts + base + lane) : 0x7fffffff;
@@ -776,6 +784,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // item, both off the softmax threads' critical path.
       const float c_scale = args.scale_log2;
       const int32_t* tb = args.table;
+      const int fs = args.fold_shift;                  // tile row m holds bin row q_row0 + (m >> fs)
       const uint32_t ring0 = (uint32_t)t * kRing;
       // row sums travel from the softmax thread to the helper of the same row, double-buffered by item
       volatile float* x_l = s_xchg + t * 128 + row;            // + 256 * (item & 1)
@@ -783,9 +792,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // key range [key_lo, key_hi] of this thread's row from a ring entry (empty for padding rows)
       // (all lanes of the warp call it together: the prompts' start rows are loaded once per warp)
       auto row_range = [&](const volatile int* e, int& key_lo, int& key_hi) {
-        const int i_row = e[4] + row;
+        const int i_row = e[4] + (row >> fs);
         int lo = e[14];
-        if (!(e[18] & 1)) lo = seg_start_at(tb + args.off_seg_start, e[16] + 1, e[13], i_row, lo, lane);
+        if (!(e[18] & 1))
+          lo = seg_start_at(tb + args.off_seg_start, e[16] + 1, e[13], i_row, e[4] + ((quad * 32 + 31) >> fs), lo, lane);
         const bool real = i_row < e[12];
         key_lo = real ? lo : 1;
         key_hi = real ? i_row : 0;
@@ -1006,7 +1016,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // until the previous store has read the staging rows.
             const uint32_t stage = s_stage_o + (uint32_t)t * Cfg::kStageOBytes + (uint32_t)quad * (32 * 128);
             const uint32_t stage_row = stage + (uint32_t)lane * 128;
-            const int p_row0 = p_q_row0 + 32 * quad;
+            const int p_row0 = p_q_row0 + ((32 * quad) >> fs);   // the warp's 32 tile rows: 32 >> fs bin rows x fold heads
 #pragma unroll 1
             for (int hh = 0; hh < D / 64; ++hh) {          // 64 columns (one TMA box) at a time
               if (lane == 0) tma_store_wait_read();
@@ -1128,7 +1138,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (used) {                                      // warp-uniform
         int lo = key_lo_t;
         if (!(single_seg & 1))                         // several prompts in this tile: find this row's
-          lo = seg_start_at(tb + args.off_seg_start, seg_first_t + 1, seg_end, i_row, lo, lane);
+          lo = seg_start_at(tb + args.off_seg_start, seg_first_t + 1, seg_end, i_row, i_row - lane + 31, lo, lane);
         if (i_row < bin_used) { key_lo = lo; key_hi = i_row; }
       }
       // Fused path: Q arrives raw and is rotated in shared memory.
@@ -1371,13 +1381,14 @@ EncodeFn get_encode_fn() {
   return fn;
 }
 
-// 4-D map over a dense [R, M, H, D] bf16 tensor; box = 64 elements x 1 head x `rows` rows x 1 bin.
-int make_map(CUtensorMap* map, const void* ptr, int64_t R, int64_t M, int64_t H, int64_t D, int rows) {
+// 4-D map over a dense [R, M, H, D] bf16 tensor; box = 64 elements x `heads` heads x `rows` rows x 1 bin
+// (in shared memory: row-major over (row, head), 128 bytes each).
+int make_map(CUtensorMap* map, const void* ptr, int64_t R, int64_t M, int64_t H, int64_t D, int rows, int heads = 1) {
   EncodeFn enc = get_encode_fn();
   if (!enc) return note_cuda_error(-1, "cuTensorMapEncodeTiled entry point not found");
   cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)M, (cuuint64_t)R};
   cuuint64_t strides[3] = {(cuuint64_t)(D * 2), (cuuint64_t)(H * D * 2), (cuuint64_t)(M * H * D * 2)};
-  cuuint32_t box[4] = {64u, 1u, (cuuint32_t)rows, 1u};
+  cuuint32_t box[4] = {64u, (cuuint32_t)heads, (cuuint32_t)rows, 1u};
   cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
   const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides,
                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1417,10 +1428,13 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   using Cfg = AttnCfg<D, BN>;
   CUtensorMap mq, mk, mv, mo;
   int st;
-  if ((st = make_map(&mq, q, p.n_bins, p.capacity, p.n_q_heads, D, BM)) != PP_OK) return st;
+  const int fold = kIndep ? L.fold : 1;
+  int fold_shift = 0;
+  while ((1 << fold_shift) < fold) ++fold_shift;
+  if ((st = make_map(&mq, q, p.n_bins, p.capacity, p.n_q_heads, D, BM / fold, fold)) != PP_OK) return st;
   if ((st = make_map(&mk, k, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
   if ((st = make_map(&mv, v, p.n_bins, p.capacity, p.n_kv_heads, D, BN)) != PP_OK) return st;
-  if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, 32)) != PP_OK) return st;   // one warp's rows per store
+  if ((st = make_map(&mo, o, p.n_bins, p.capacity, p.n_q_heads, D, 32 / fold, fold)) != PP_OK) return st;   // one warp's rows per store
   // the shared-memory opt-in of a kernel is a per-device attribute
   static DeviceOnce configured;     // per template instance
   int dev = 0;
@@ -1443,7 +1457,9 @@ int launch_attention_t(const pp_attn_params& p, int32_t* d_table, const TableLay
   a.n_items = L.n_items;
   a.group = p.n_q_heads / p.n_kv_heads;
   a.pair_heads = (!kIndep && a.group % 2 == 0) ? 1 : 0;
-  a.subs = a.pair_heads ? a.group / 2 : a.group;
+  a.fold = fold;
+  a.fold_shift = fold_shift;
+  a.subs = a.pair_heads ? a.group / 2 : a.group / fold;
   a.n_q_heads = p.n_q_heads;
   a.capacity = p.capacity;
   const int64_t total = (int64_t)p.n_kv_heads * L.n_items * a.subs;

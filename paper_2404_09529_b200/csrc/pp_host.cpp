@@ -173,8 +173,16 @@ extern "C" int pp_fill_position_ids(int32_t n_bins, int32_t capacity, const int3
 // ------------------------------------------------------------------------------------------
 namespace pp {
 
-size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k) {
-  const int64_t q_tiles = (int64_t)n_bins * ((capacity + kTileM - 1) / kTileM);
+int32_t max_fold(int32_t group) {
+  for (int32_t f = kMaxFold; f > 1; f >>= 1)
+    if (group % f == 0) return f;
+  return 1;
+}
+
+size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k, int32_t group) {
+  // sized for the shortest query tiles any mode can choose (head folding shortens them)
+  const int32_t rq = kTileM / max_fold(group);
+  const int64_t q_tiles = (int64_t)n_bins * ((capacity + rq - 1) / rq);
   // header + bin_seg_ptr + bin_used + seg_start + items (kItemInts ints each), each block 4-int aligned
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
   return (size_t)(kHeaderInts + up4(n_bins + 1) + up4(n_bins) + up4(k) + kItemInts * q_tiles);
@@ -213,13 +221,18 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   const bool independent = mean_key_tiles(n_bins, bin_seg_ptr, seg_start, seg_len) < 8.0;
   const bool pair_rows = !even_group && !independent;
   const int32_t tile_n = independent ? kTileNShort : kTileN;   // key rows per tile of the chosen mode
+  //  - short items and several query heads per KV head: the heads are folded into the rows of a
+  //    query tile (128 / fold rows x fold heads), so one stream of key tiles serves all of them and a
+  //    short prompt fills a tile with heads instead of leaving most of its rows empty
+  const int32_t fold = independent ? max_fold(group) : 1;
+  const int32_t rq = kTileM / fold;                            // bin rows per query tile
   auto up4 = [](int64_t x) { return (x + 3) & ~int64_t(3); };
   TableLayout L;
   L.bin_seg_ptr = kHeaderInts;
   L.bin_used = L.bin_seg_ptr + (int32_t)up4(n_bins + 1);
   L.seg_start = L.bin_used + (int32_t)up4(n_bins);
   L.items = L.seg_start + (int32_t)up4(k);
-  if (out_ints < prefill_table_ints(n_bins, capacity, k)) return PP_ERR_BUFFER_TOO_SMALL;
+  if (out_ints < prefill_table_ints(n_bins, capacity, k, group)) return PP_ERR_BUFFER_TOO_SMALL;
   std::memset(out, 0, sizeof(int32_t) * (size_t)L.items);
   std::memcpy(out + L.bin_seg_ptr, bin_seg_ptr, sizeof(int32_t) * (size_t)(n_bins + 1));
   std::memcpy(out + L.seg_start, seg_start, sizeof(int32_t) * (size_t)k);
@@ -229,13 +242,14 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
       const int32_t s_lo = bin_seg_ptr[b], s_hi = bin_seg_ptr[b + 1];
       const int32_t used = seg_start[s_hi - 1] + seg_len[s_hi - 1];
       out[L.bin_used + b] = used;
-      int32_t s = s_lo;
-      // first key row (rounded down to a key tile) that query tile q0 can see
+      int32_t s = s_lo, s_slot0 = s_lo;     // cursors over the bin's segments: query rows only move forward
+      // first key row that query tile q0 can see: the start of the prompt that holds row q0, rounded
+      // down to a key tile where two slots share the stream (their tiles must coincide)
       auto kv_lo_of = [&](int32_t q0) {
         while (s + 1 < s_hi && seg_start[s + 1] <= q0) ++s;       // segment holding row q0
-        return (seg_start[s] / tile_n) * tile_n;
+        return independent ? seg_start[s] : (seg_start[s] / tile_n) * tile_n;
       };
-      const int32_t step = pair_rows ? 2 * kTileM : kTileM;
+      const int32_t step = pair_rows ? 2 * kTileM : rq;
       for (int32_t q0 = 0; q0 < used; q0 += step) {
         WorkItem it{};
         it.bin = b;
@@ -243,7 +257,7 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
         it.q_row0[0] = q0;
         if (!pair_rows) {                       // two heads, same rows
           it.q_row0[1] = q0;
-          it.n_kv_tiles = (std::min(q0 + kTileM, used) - it.kv_row0 + tile_n - 1) / tile_n;
+          it.n_kv_tiles = (std::min(q0 + rq, used) - it.kv_row0 + tile_n - 1) / tile_n;
           it.jb1 = 0;
           it.je0 = it.n_kv_tiles;
         } else if (q0 + kTileM < used) {        // two consecutive row tiles
@@ -264,11 +278,13 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
         for (int t = 0; t < 2; ++t) {
           const int32_t q = it.q_row0[t];
           if (q < 0) continue;
-          int32_t sf = s_lo;                    // segment holding row q (bins hold few segments)
+          // segment holding row q: slot 0's rows ascend from item to item, slot 1 starts from slot 0's
+          int32_t sf = s_slot0;
           while (sf + 1 < s_hi && seg_start[sf + 1] <= q) ++sf;
+          if (t == 0) s_slot0 = sf;
           it.seg_first[t] = sf;
           it.key_lo[t] = seg_start[sf];
-          const int32_t last_row = std::min(q + kTileM, used) - 1;
+          const int32_t last_row = std::min(q + rq, used) - 1;
           if (sf + 1 >= s_hi || seg_start[sf + 1] > last_row) it.single_seg |= 1 << t;
         }
         items.push_back(it);
@@ -300,6 +316,7 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   L.total_ints = (int32_t)(L.items + kItemInts * (int64_t)items.size());
   L.independent_slots = independent;
   L.pair_rows = pair_rows;
+  L.fold = fold;
   if (layout) *layout = L;
   return PP_OK;
 }
@@ -315,10 +332,11 @@ extern "C" int pp_prefill_schedule_info(const pp_attn_params* params, const int3
   int st = pp::validate_packing(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k);
   if (st != PP_OK) return st;
   try {
-    std::vector<int32_t> table(pp::prefill_table_ints(params->n_bins, params->capacity, k));
+    const int32_t group = params->n_q_heads / params->n_kv_heads;
+    std::vector<int32_t> table(pp::prefill_table_ints(params->n_bins, params->capacity, k, group));
     pp::TableLayout L;
     st = pp::build_prefill_tables(params->n_bins, params->capacity, bin_seg_ptr, seg_start, seg_len, k,
-                                  params->n_q_heads / params->n_kv_heads, table.data(), table.size(), &L);
+                                  group, table.data(), table.size(), &L);
     if (st != PP_OK) return st;
     const pp::WorkItem* items = reinterpret_cast<const pp::WorkItem*>(table.data() + L.items);
     int64_t steps = 0;
@@ -335,7 +353,7 @@ extern "C" int pp_prefill_schedule_info(const pp_attn_params* params, const int3
     info[4] = L.independent_slots ? pp::kTileNShort : pp::kTileN;
     info[5] = unpaired;
     info[6] = late;
-    info[7] = 1;
+    info[7] = L.fold;
   } catch (const std::bad_alloc&) {
     return PP_ERR_NO_MEMORY;
   }

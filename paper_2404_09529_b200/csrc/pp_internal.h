@@ -15,6 +15,7 @@ constexpr int kTileNShort = 64;  // the same in independent-slot mode (short wor
 constexpr int kHeaderInts = 16;  // table header, see build_prefill_tables
 constexpr int kHeaderCounter = 10;   // header word the persistent CTAs draw work indices from
 constexpr int kItemInts = 16;
+constexpr int kMaxFold = 8;      // most query heads of one KV head folded into the rows of a query tile
 
 // One entry of the attention work list: two query-tile slots sharing one key/value tile stream.
 struct WorkItem {
@@ -44,11 +45,13 @@ struct TableLayout {
   int32_t total_ints = 0;
   bool independent_slots = false;   // items are single tiles, drawn by each slot on its own
   bool pair_rows = false;           // shared-stream mode: the two slots are consecutive row tiles of one head
+  int32_t fold = 1;                 // independent mode: query heads folded into a query tile (128 / fold bin rows each)
 };
 
 int validate_packing(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
                      const int32_t* seg_start, const int32_t* seg_len, int32_t k);
-size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k);
+size_t prefill_table_ints(int32_t n_bins, int32_t capacity, int32_t k, int32_t group);
+int32_t max_fold(int32_t group);   // largest power of two <= kMaxFold that divides the GQA group
 int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_seg_ptr,
                          const int32_t* seg_start, const int32_t* seg_len, int32_t k, int32_t group,
                          int32_t* out, size_t out_ints, TableLayout* layout);
