@@ -142,11 +142,25 @@ def whole_job_tokens_per_s(world: int, tokens_per_rank: int, ms_per_step: float)
     return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
+_FLUSH = None      # set by main() for workloads smaller than the L2: a buffer to overwrite before every timed call
+
+
 def time_loop(fn, iters, warmup=3):
     import torch
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
+    if _FLUSH is not None:
+        # small workload: every call is timed on its own, after the L2 has been overwritten; the flush
+        # kernel also gives the host the time to queue the call, so the events bracket device time
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        for a, b in evs:
+            _FLUSH.fill_(1)
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in evs) / iters
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     # A few milliseconds of device-side delay in front of the first event let the host queue all the
     # calls before the first one starts, so the events bracket launches that run back to back: the
@@ -199,7 +213,7 @@ def workload_config(cfg, name, lengths, n_bins, capacity, world):
     stream_mb = (rows * d * 2 * (2 * hq + 3 * hkv) + T * d * 2 * 2 * hkv) / 1e6
     l2 = (f"no flush: each step streams {stream_mb:.0f} MB of tensors, larger than the 126 MB L2"
           if stream_mb > 2 * 126 else
-          f"flushed: each step touches only {stream_mb:.1f} MB, so a 256 MB buffer is overwritten before every "
+          f"flushed: each step touches only {stream_mb:.1f} MB, so a 1 GB buffer is overwritten before every "
           "timed step and the steps are timed one by one")
     return {"workload": name, "description": cfg.description, "n_prompts": int(len(lengths)),
             "total_tokens": T, "n_bins": int(n_bins), "capacity": int(capacity),
@@ -308,8 +322,12 @@ def main():
     routes = {"three_call": lambda: batch.run(repack=True), "fused": lambda: batch.run_fused(repack=True)}
     config, stream_mb = workload_config(cfg, args.workload, lengths, batch.pack.n_bins, batch.pack.capacity, world)
     # A step that touches less than about twice the L2 would find its inputs there on the next step:
-    # such workloads are timed step by step, with a 256 MB buffer overwritten before each.
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if stream_mb <= 2 * 126 else None
+    # such workloads are timed step by step, with a 1 GB buffer overwritten before each.
+    # (1 GB rather than just more than the L2: the overwrite must also outlast the host's enqueueing
+    # of the step behind it, or the events would bracket host time)
+    flush = torch.empty(1 << 30, dtype=torch.uint8, device="cuda") if stream_mb <= 2 * 126 else None
+    global _FLUSH
+    _FLUSH = flush
 
     def timed_region(step):
         batch.load(q_tok, k_tok, v_tok)          # raw Q/K again (the three-call route rotates q in place)
