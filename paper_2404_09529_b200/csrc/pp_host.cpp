@@ -71,10 +71,20 @@ extern "C" int pp_pack(const int32_t* lengths, int32_t k, int32_t capacity, int3
   const int32_t cap = capacity == 0 ? longest : capacity;
   if (longest > cap) return PP_ERR_LENGTH;
   try {
+    // items by length descending, equal lengths by original index ascending: a counting sort over
+    // the lengths (they are at most `cap`), falling back to a comparison sort for few long prompts
     std::vector<int32_t> order(k);
-    std::iota(order.begin(), order.end(), 0);
-    std::stable_sort(order.begin(), order.end(),
-                     [&](int32_t a, int32_t b) { return lengths[a] > lengths[b]; });
+    if ((int64_t)longest <= 8 * (int64_t)k + 1024) {
+      std::vector<int32_t> first(longest + 2, 0);             // first[l] = items longer than l, so far: counts
+      for (int32_t i = 0; i < k; ++i) ++first[lengths[i]];
+      int32_t run = 0;
+      for (int32_t l = longest; l >= 1; --l) { const int32_t c = first[l]; first[l] = run; run += c; }
+      for (int32_t i = 0; i < k; ++i) order[first[lengths[i]]++] = i;
+    } else {
+      std::iota(order.begin(), order.end(), 0);
+      std::stable_sort(order.begin(), order.end(),
+                       [&](int32_t a, int32_t b) { return lengths[a] > lengths[b]; });
+    }
     FirstFitTree tree(k);
     std::vector<int32_t> item_bin(k), item_off(k), bin_count;
     int32_t r = 0;
@@ -238,6 +248,7 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
   std::memcpy(out + L.seg_start, seg_start, sizeof(int32_t) * (size_t)k);
   std::vector<WorkItem> items;
   try {
+    items.reserve((size_t)n_bins * ((capacity + rq - 1) / rq));
     for (int32_t b = 0; b < n_bins; ++b) {
       const int32_t s_lo = bin_seg_ptr[b], s_hi = bin_seg_ptr[b + 1];
       const int32_t used = seg_start[s_hi - 1] + seg_len[s_hi - 1];
@@ -291,9 +302,18 @@ int build_prefill_tables(int32_t n_bins, int32_t capacity, const int32_t* bin_se
       }
     }
     // Longest first: CTAs draw items in list order, which gives longest-processing-time-first
-    // scheduling; ties keep bin/row order.
-    std::stable_sort(items.begin(), items.end(),
-                     [](const WorkItem& a, const WorkItem& b) { return a.cost > b.cost; });
+    // scheduling; ties keep bin/row order (a stable counting sort over the costs).
+    {
+      int32_t max_cost = 0;
+      for (const WorkItem& it : items) max_cost = std::max(max_cost, it.cost);
+      std::vector<int32_t> first(max_cost + 2, 0);
+      for (const WorkItem& it : items) ++first[it.cost];
+      int32_t run = 0;
+      for (int32_t c = max_cost; c >= 0; --c) { const int32_t n = first[c]; first[c] = run; run += n; }
+      std::vector<WorkItem> sorted(items.size());
+      for (const WorkItem& it : items) sorted[first[it.cost]++] = it;
+      items.swap(sorted);
+    }
   } catch (const std::bad_alloc&) {
     return PP_ERR_NO_MEMORY;
   }
