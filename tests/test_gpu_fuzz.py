@@ -27,6 +27,38 @@ def _draw(rng):
     return lengths.astype(np.int32), hq, hkv, d, float(rng.choice([10000.0, 500000.0]))
 
 
+def _draw_long(rng):
+    """A few long prompts next to short ones: the shared-stream mode of the attention kernel, with head
+    pairs (even GQA group) or paired row tiles (odd group), tile counts odd and even."""
+    d = int(rng.choice([64, 128]))
+    hkv = int(rng.choice([1, 2]))
+    hq = hkv * int(rng.choice([1, 2, 3]))
+    lengths = np.concatenate([rng.integers(1400, 3300, size=int(rng.integers(1, 4))),
+                              rng.integers(1, 200, size=int(rng.integers(0, 6)))])
+    return lengths.astype(np.int32), hq, hkv, d, float(rng.choice([10000.0, 500000.0]))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_long_shapes_full_parity(seed):
+    rng = np.random.default_rng(5000 + seed)
+    lengths, hq, hkv, d, base = _draw_long(rng)
+    t = int(lengths.sum())
+    gen = torch.Generator().manual_seed(100 + seed)
+    q = torch.randn(t, hq, d, generator=gen).to(torch.bfloat16)
+    k = torch.randn(t, hkv, d, generator=gen).to(torch.bfloat16)
+    v = torch.randn(t, hkv, d, generator=gen).to(torch.bfloat16)
+    from parity_utils import compare_with_refs, oracle_refs
+    refs = oracle_refs(lengths, q, k, v, base)
+    for fused in (False, True):
+        b = PrefillBatch(lengths, hq, hkv, d, base, guard=True)
+        b.load(q, k, v)
+        b.run_fused() if fused else b.run()
+        torch.cuda.synchronize()
+        assert b.device_status() == 0
+        b.assert_untouched()
+        compare_with_refs(b, lengths, refs)
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_random_shapes_full_parity(seed):
     rng = np.random.default_rng(1000 + seed)

@@ -75,6 +75,34 @@ def test_shared_stream_variants_full_parity(lengths, hq, hkv, d, pairing, unpair
             compare_with_refs(b, lengths, refs)
 
 
+# lengths, Hq, Hkv, D, query heads folded into a query tile (independent mode: the largest of 8, 4, 2
+# that divides the GQA group; 1 = MHA or an odd group)
+FOLD_CASES = [
+    ([129, 1, 1, 127, 40, 3], 2, 1, 64, 2),
+    ([300, 5, 129, 64, 1, 250, 33, 8, 8, 8, 90, 2], 8, 2, 128, 4),
+    ([515, 130, 129, 128, 64, 33, 17, 9, 3, 2, 1], 8, 1, 64, 8),
+    ([8] * 40 + [31, 33, 65], 16, 1, 128, 8),                  # group 16: two folds of 8 per KV head
+    ([200, 77, 130, 31, 12], 6, 2, 64, 1),                     # group 3: no fold
+    ([200, 77, 130, 31, 12], 12, 2, 128, 2),                   # group 6: folds of 2
+]
+
+
+@pytest.mark.parametrize("lengths,hq,hkv,d,fold", FOLD_CASES)
+def test_head_folding_variants_full_parity(lengths, hq, hkv, d, fold):
+    """Independent mode with GQA: the query tile is 128 / fold bin rows x fold heads. Every fold the
+    scheduler can choose, both batch modes, both routes, guard regions around every output."""
+    lengths = np.asarray(lengths, np.int32)
+    base = 10000.0
+    q, k, v = _case(lengths, hq, hkv, d, seed=hq * 100 + d)
+    refs = oracle_refs(lengths, q, k, v, base)
+    for mode in ("packed", "padded"):
+        for fused in (False, True):
+            b = run_cuda(lengths, q, k, v, hq, hkv, d, base, mode, fused=fused, guard=True)
+            info = pp.pp_prefill_schedule_info(b.params, b.pack)
+            assert info["mode"] == 1 and info["heads_folded"] == fold, info
+            compare_with_refs(b, lengths, refs)
+
+
 @pytest.mark.parametrize("room", [1, 7, 64])
 @pytest.mark.parametrize("lengths,hq,hkv,d", [
     ([112, 87, 73, 46, 50, 20, 24, 17], 4, 4, 64),          # several prompts per bin, independent mode
