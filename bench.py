@@ -31,9 +31,10 @@ METRIC = "useful_prefill_tokens_per_s"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "llama2_7b"
 
-# DRAM traffic of one attention-kernel launch on the fused route (dram__bytes_read.sum +
-# dram__bytes_write.sum) from the ncu captures summarised in profiles/attention_<workload>.md; None
-# where no capture exists for the workload.
+# DRAM traffic of one attention-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) from
+# the ncu captures summarised in profiles/attention_<workload>.md (fused-route launches; long_mix: a
+# launch of the three-call route, which reads and writes the same tensors); None where no capture
+# exists for the workload.
 NCU_ATTENTION_TRAFFIC_BYTES = {"llama2_7b": 562.4e6, "many_short": 424.2e6, "long_mix": 3.82e9}
 
 
