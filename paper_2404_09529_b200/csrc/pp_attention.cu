@@ -699,6 +699,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         if (t == 1 || !(j >= jb1 && j < je1)) tc_commit(bar_k_empty + 8 * s);
         tc_commit(bar_s_full + 16 * t);
+        // the slot's last scores of this item: its Q buffer is free for the next item's Q from here on
+        if (j + 1 == (t ? je1 : je0)) tc_commit(bar_q_empty + 8 * t);
         return true;
       };
       // O_t (+)= P_t V_j, then either the next S_t or the end-of-item signals of slot t
@@ -721,8 +723,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           ++tcount;
           if (t == 1 || !(j >= jb1 && j < je1)) tc_commit(bar_v_empty + 8 * s);
           if (j + 1 < je) return issue_qk(t, j + 1);
-          tc_commit(bar_q_empty + 8 * t);      // slot t is done with this item
-          tc_commit(bar_o_full + 8 * t);
+          tc_commit(bar_o_full + 8 * t);       // slot t is done with this item
           return true;
         }
         if (j + 1 == jb && jb < je) return issue_qk(t, j + 1);   // slot t joins the key loop at the next tile
