@@ -185,13 +185,15 @@ int pp_prefill_attention(const pp_attn_params* params,
  *   v, o         as in pp_prefill_attention
  *   k_cache, v_cache, cache_off, cache_cap   as in pp_unpack_kv (original prompt order)
  *   workspace    device, >= pp_prefill_fused_workspace_bytes, 256-byte aligned (tables and a
- *                cos/sin table of capacity * D/2 pairs); host_workspace: host staging of the same
- *                size or at least the table part, pinned memory keeps the call asynchronous
+ *                cos/sin table of capacity * D/2 pairs); host_workspace: host staging of at least
+ *                pp_prefill_fused_host_bytes (the tables, which are what is uploaded; the cos/sin
+ *                table is built on the device), pinned memory keeps the call asynchronous
  * params->flags: PP_FLAG_ROPE_ONLY runs only the rotation / unpack kernels, PP_FLAG_SKIP_ROPE only the
  * attention kernel (k_ holds rotated keys already). Outputs are bit-identical to the two-call path.
  * Errors as the two calls it replaces.
  */
 size_t pp_prefill_fused_workspace_bytes(const pp_attn_params* params, int32_t k);
+size_t pp_prefill_fused_host_bytes(const pp_attn_params* params, int32_t k);
 int pp_prefill_fused(const pp_attn_params* params,
                      const int32_t* bin_seg_ptr, const int32_t* seg_start, const int32_t* seg_len,
                      const int32_t* seg_prompt, int32_t k, const int32_t* lengths,

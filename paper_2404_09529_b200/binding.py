@@ -60,6 +60,7 @@ def load_library():
         "pp_prefill_attention": (ctypes.c_int, [pp, i32p, i32p, i32p, ctypes.c_int32, vp, vp, vp, vp, vp, vp,
                                                 ctypes.c_size_t, vp, vp]),
         "pp_prefill_fused_workspace_bytes": (ctypes.c_size_t, [pp, ctypes.c_int32]),
+        "pp_prefill_fused_host_bytes": (ctypes.c_size_t, [pp, ctypes.c_int32]),
         "pp_prefill_fused": (ctypes.c_int, [pp, i32p, i32p, i32p, i32p, ctypes.c_int32, i32p, vp, vp, vp, vp, vp, vp,
                                             i64p, i32p, vp, vp, ctypes.c_size_t, vp, vp]),
         "pp_selftest_bounded_wait": (ctypes.c_int, [vp, ctypes.c_uint32, vp]),
@@ -194,6 +195,10 @@ def pp_prefill_fused_workspace_bytes(params: AttnParams, k: int) -> int:
     return int(load_library().pp_prefill_fused_workspace_bytes(ctypes.byref(params), k))
 
 
+def pp_prefill_fused_host_bytes(params: AttnParams, k: int) -> int:
+    return int(load_library().pp_prefill_fused_host_bytes(ctypes.byref(params), k))
+
+
 def pp_prefill_fused(params: AttnParams, pack: Packing, lengths, q, k, v, o, k_cache, v_cache, cache_off,
                      cache_cap, workspace, host_workspace, workspace_bytes: int, device_status=None,
                      stream: int = 0) -> None:
@@ -305,7 +310,7 @@ class Workspaces:
         self.attn_dev = torch.empty(self.attn_bytes, dtype=torch.uint8, device=device)
         self.unpack_dev = torch.empty(self.unpack_bytes, dtype=torch.uint8, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
-        self._fused_host = [torch.empty(self.attn_bytes + 32 * k + 256, dtype=torch.uint8).pin_memory()
+        self._fused_host = [torch.empty(pp_prefill_fused_host_bytes(params, k), dtype=torch.uint8).pin_memory()
                             for _ in range(ring)]
         self._ring = [(torch.empty(self.attn_bytes, dtype=torch.uint8).pin_memory(),
                        torch.empty(self.unpack_bytes, dtype=torch.uint8).pin_memory(),

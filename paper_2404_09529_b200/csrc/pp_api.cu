@@ -143,6 +143,11 @@ extern "C" size_t pp_prefill_fused_workspace_bytes(const pp_attn_params* params,
   return pp::fused_layout(*params, k).total_bytes;
 }
 
+extern "C" size_t pp_prefill_fused_host_bytes(const pp_attn_params* params, int32_t k) {
+  if (pp::check_params(params) != PP_OK || k < 1) return 0;
+  return sizeof(int32_t) * pp::fused_layout(*params, k).upload_ints;
+}
+
 namespace pp {
 namespace {
 // The kernels of the fused path on tables that are (or will be, in stream order) in `workspace`.
